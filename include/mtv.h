@@ -1,0 +1,229 @@
+/*
+ * mtv.h — C ABI of the static-tree verification library (Medusa-style
+ * speculative decoding, one verification step on one NVIDIA B200, sm_100a).
+ *
+ * One decode step (Section 3.1 and Section 3.2 of the paper):
+ *   medusa_heads_topk      K residual-MLP heads -> per-head top-k -> flat candidate
+ *                          buffer -> tokens of the T static tree nodes
+ *   tree_verify_attention  attention of all T tree nodes over [prefix ; tree] K/V under
+ *                          the static visibility matrix (once per backbone layer)
+ *   tree_accept            greedy longest-prefix acceptance + Gather of the accepted
+ *                          tokens through retrieve_indices
+ *   kv_compact_accepted    the same Gather applied to the accepted nodes' K/V rows,
+ *                          in place, all layers; advances seq_lens
+ * with the tree's static tensors built once by tree_build_static.
+ *
+ * Conventions
+ *   - Every function returns an int: MTV_OK (0) or a negative MTV_ERR_* code.
+ *   - "device" pointers are CUDA global-memory addresses valid on the current
+ *     device; "host" pointers are ordinary process memory.  The caller owns every
+ *     buffer; the library owns only mtv_tree_t objects.
+ *   - Hot calls (the four step functions and mtv_verify_step) only enqueue work on
+ *     `stream` (a cudaStream_t passed as void*; NULL = default stream).  They never
+ *     allocate, never synchronise and never copy to the host.  Results are ready
+ *     when the stream reaches the end of the enqueued work.
+ *   - bf16 data is passed as raw 16-bit patterns (mtv_bf16).  Indices are int32.
+ *   - Data-dependent faults (a sequence that does not fit its cache) are written to
+ *     the caller's device `status[B]` (0 = ok, MTV_ERR_* otherwise); the outputs of
+ *     that sequence are left untouched.  status may be NULL.
+ *   - Supported shapes: D in {64, 128}; 1 <= T <= 128; 1 <= K <= 8; per-depth
+ *     top-k <= 16; Hq a multiple of Hkv with Hq/Hkv <= 8; H a multiple of 8.
+ *     Anything else returns MTV_ERR_UNSUPPORTED_SHAPE.
+ */
+#ifndef MTV_H_
+#define MTV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MTV_OK 0
+#define MTV_ERR_INVALID_ARG (-1)
+#define MTV_ERR_UNSUPPORTED_SHAPE (-2)
+#define MTV_ERR_WORKSPACE (-3)
+#define MTV_ERR_CUDA (-4)
+#define MTV_ERR_TIMEOUT (-5)
+#define MTV_ERR_CAPACITY (-6) /* status[b]: seq_lens[b] + T exceeds the cache capacity */
+
+#define MTV_MAX_K 8
+#define MTV_MAX_T 128
+#define MTV_MAX_TOPK 16
+
+typedef uint16_t mtv_bf16;
+typedef struct mtv_tree mtv_tree_t;
+
+/* Host view of a tree's static tensors (pointers stay valid until tree_destroy). */
+typedef struct {
+    int32_t T;           /* nodes including the root */
+    int32_t K;           /* heads = maximum depth */
+    int32_t P;           /* N_paths = number of leaves */
+    int32_t C;           /* flat candidate buffer length = 1 + sum k_d */
+    int32_t anc_words;   /* 64-bit words per row of anc */
+    int32_t on_device;   /* 1 if the tables were uploaded */
+    int32_t k_d[MTV_MAX_K];         /* candidates taken from head d+1 */
+    int32_t cand_offset[MTV_MAX_K]; /* first slot of head d+1 in the candidate buffer */
+    const int32_t *node_ranks;       /* [T][K] rank tuple of each node, -1 padded */
+    const int32_t *parent;           /* [T], -1 for the root */
+    const int32_t *depth;            /* [T] */
+    const int32_t *rank;             /* [T] rank within its head, -1 for the root */
+    const int32_t *tree_indices;     /* [T] node -> slot of the candidate buffer */
+    const int32_t *retrieve_indices; /* [P][K+1] node ids root..leaf, -1 padded */
+    const uint64_t *anc;             /* [T][anc_words] ancestor-or-self bitmask */
+    const uint8_t *medusa_attn_mask; /* [T][T] dense 0/1 form of anc */
+} mtv_tree_info;
+
+/* ---------------------------------------------------------------------------
+ * Static tree tensors — Section 3.2, "Tensorization of Tree Topology" (the
+ * visibility matrix medusa_attn_mask and tree_indices) and "Zero-Copy Retrieval"
+ * (retrieve_indices [N_paths][K+1]).  Host-side, run once at initialisation.
+ *
+ * node_ranks: host, [n_nodes][K] int32.  Row = the per-depth ranks on the way from
+ *   the root to the node (r_1..r_d), padded with -1.  The root is implicit.  Order is
+ *   free; duplicates are an error; every node's parent must be present.
+ * The flattened order is root first, then ascending (depth, rank tuple).  Node i's
+ *   K/V row lives in cache slot seq_lens[b] + i; its token is candidate slot
+ *   tree_indices[i]; paths are ordered by ascending leaf index.
+ * upload != 0 copies the tables to the current CUDA device (needed by the hot
+ *   calls); upload == 0 builds the host tables only (no CUDA call is made).
+ * Errors: MTV_ERR_INVALID_ARG (bad ranks, orphan, duplicate), MTV_ERR_UNSUPPORTED_SHAPE
+ *   (K, T or a top-k beyond the limits), MTV_ERR_CUDA (upload failed).
+ */
+int tree_build_static(int K, int n_nodes, const int32_t *node_ranks, int upload, mtv_tree_t **out);
+
+/* Full Cartesian tree: every rank tuple with r_d < topk[d].  node_ranks: host
+ * [capacity][K]; *n_nodes receives the node count (root excluded).  Returns
+ * MTV_ERR_INVALID_ARG if capacity is too small (then *n_nodes = needed count). */
+int tree_gen_cartesian(int K, const int32_t *topk, int capacity, int32_t *node_ranks, int *n_nodes);
+
+/* Sparse tree: root plus the T_total-1 highest-scoring nodes of the full R_max-ary
+ * depth-K tree, score = product over depths of p(r) = 1/((r+1) Z), Z = sum_{r<R_max} 1/(r+1);
+ * ties by depth ascending then rank tuple ascending; scores compared exactly.
+ * node_ranks: host [T_total-1][K].  R_max <= 16, K <= 7. */
+int tree_gen_rank_prior(int K, int T_total, int R_max, int32_t *node_ranks, int *n_nodes);
+
+int tree_query(const mtv_tree_t *tree, mtv_tree_info *info);
+void tree_destroy(mtv_tree_t *tree);
+
+/* Bytes of device scratch that any hot call below may need for these shapes.
+ * Lcap = cache capacity in rows.  The same buffer may be reused by successive
+ * calls on one stream; concurrent calls need separate buffers.  Returns 0 on
+ * invalid arguments. */
+size_t mtv_workspace_bytes(const mtv_tree_t *tree, int B, int H, int V, int Hq, int Hkv, int D, int Lcap);
+
+/* ---------------------------------------------------------------------------
+ * Medusa heads + per-head top-k + tree expansion — Section 3.1 (K parallel heads,
+ * each an MLP with a residual connection, head k predicting token t+k+1) and the
+ * candidate buffer of Section 3.2.
+ *   y = W1_k h_b + b1_k;  h' = h_b + SiLU(y);  z_k = W2_k h'      (fp32, no rounding between)
+ *   cand[b] = [root_tok[b] | ids of the k_1 largest z_1 | k_2 largest z_2 | ...]
+ *             (descending logit, equal logits by ascending id)
+ *   tree_tok[b][i] = cand[b][tree_indices[i]]
+ * All pointers device.  hidden [B][H]; W1 [K][H][H] and W2 [K][V][H] row-major with
+ * the output feature outermost; b1 [K][H] or NULL; root_tok [B]; cand [B][C];
+ * cand_logit [B][C-1] fp32 or NULL; tree_tok [B][T].  1 <= B <= 16.
+ */
+int medusa_heads_topk(const mtv_tree_t *tree, int B, int H, int V,
+                      const mtv_bf16 *hidden, const mtv_bf16 *W1, const mtv_bf16 *b1,
+                      const mtv_bf16 *W2, const int32_t *root_tok,
+                      int32_t *cand, float *cand_logit, int32_t *tree_tok,
+                      void *ws, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * Tree attention — Section 3.2 / Fig. 2(b): the T tree nodes attend to the KV cache
+ * under the static visibility matrix.  For sequence b, node i, query head h
+ * (KV head g = h / (Hq/Hkv)):
+ *   visible = [0, seq_lens[b])  U  { seq_lens[b] + a : a ancestor-or-self of i }
+ *   out[b][i][h] = softmax_j(scale <q[b][i][h], k[b][g][j]>) . v[b][g][j]   over visible j
+ * bf16 inputs, fp32 scores / softmax / accumulation, bf16 output (round to nearest even).
+ * All pointers device.  q, out [B][T][Hq][D] contiguous.  k_cache / v_cache: element
+ * (b, g, row, d) at b*stride_b + g*stride_h + row*stride_t + d (strides in elements,
+ * multiples of 8; base 16-byte aligned); the caller has already written the tree
+ * nodes' K/V to rows seq_lens[b] + i.  seq_lens [B] device int32 (0 is legal).
+ * scale == 0 means 1/sqrt(D).  status[b] = MTV_ERR_CAPACITY if seq_lens[b] + T > Lcap.
+ */
+int tree_verify_attention(const mtv_tree_t *tree, int B, int Hq, int Hkv, int D,
+                          const mtv_bf16 *q, const mtv_bf16 *k_cache, const mtv_bf16 *v_cache,
+                          int64_t stride_b, int64_t stride_h, int64_t stride_t, int Lcap,
+                          const int32_t *seq_lens, float scale,
+                          mtv_bf16 *out, int32_t *status,
+                          void *ws, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * Acceptance + token retrieval — Section 3.2, "Zero-Copy Retrieval": the best path
+ * index is found by the acceptance criterion and the final token sequence is
+ * gathered from the candidates through retrieve_indices, all on the device.
+ *   am[b][i]  = argmax_v logits[b][i][v]                        (ties: lowest v)
+ *   len_p     = number of leading j >= 1 with tree_tok[b][ri[p][j]] == am[b][ri[p][j-1]]
+ *   best_path = argmax_p len_p (ties: lowest p);  accept_len = len_best in [0, K]
+ *   acc_nodes[b][0..accept_len] = ri[best][..], acc_tok = tree_tok at those nodes, -1 padded
+ *   next_root[b] = am[b][acc_nodes[b][accept_len]]
+ * All pointers device.  logits [B][T][V] bf16 (base-model logits at every tree node).
+ * Outputs: accept_len, best_path, next_root [B]; acc_nodes, acc_tok [B][K+1].
+ */
+int tree_accept(const mtv_tree_t *tree, int B, int V, const mtv_bf16 *logits, const int32_t *tree_tok,
+                int32_t *accept_len, int32_t *best_path, int32_t *acc_nodes, int32_t *acc_tok,
+                int32_t *next_root, void *ws, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * KV compaction — Section 3.2, "Zero-Copy Retrieval" applied to K/V: for every layer,
+ * sequence b, KV head g and j = 1..accept_len[b], row seq_lens[b] + acc_nodes[b][j]
+ * moves to row seq_lens[b] + j, in place (all sources are read before any row is
+ * written); then seq_lens[b] += accept_len[b] + 1.
+ * k_caches / v_caches: device arrays of n_layers device pointers, every cache with
+ * the strides of tree_verify_attention.  seq_lens is read and updated on the device.
+ * status[b] = MTV_ERR_CAPACITY (and b is skipped) if seq_lens[b] + T > Lcap.
+ */
+int kv_compact_accepted(const mtv_tree_t *tree, int B, int Hkv, int D, int n_layers,
+                        mtv_bf16 *const *k_caches, mtv_bf16 *const *v_caches,
+                        int64_t stride_b, int64_t stride_h, int64_t stride_t, int Lcap,
+                        int32_t *seq_lens, const int32_t *accept_len, const int32_t *acc_nodes,
+                        int32_t *status, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * One whole verification step (the order of Section 3.2's pipeline), enqueued on
+ * one stream with no host involvement: heads -> attention for each of n_layers
+ * caches -> acceptance -> compaction.  Device pointers throughout.
+ * q_layers / out_layers: [n_layers][B][T][Hq][D] contiguous.
+ */
+typedef struct {
+    int32_t B, H, V, Hq, Hkv, D, n_layers, Lcap;
+    int64_t stride_b, stride_h, stride_t;
+    float scale;
+    const mtv_bf16 *hidden, *W1, *b1, *W2;
+    const int32_t *root_tok;
+    const mtv_bf16 *q_layers;
+    mtv_bf16 *const *k_caches; /* device array [n_layers] */
+    mtv_bf16 *const *v_caches; /* device array [n_layers] */
+    mtv_bf16 *const *k_caches_host; /* host copy of the same pointer array */
+    mtv_bf16 *const *v_caches_host;
+    const mtv_bf16 *logits;    /* [B][T][V] */
+    int32_t *seq_lens;         /* [B] in/out */
+    int32_t *cand; float *cand_logit; int32_t *tree_tok;
+    mtv_bf16 *out_layers;
+    int32_t *accept_len, *best_path, *acc_nodes, *acc_tok, *next_root;
+    int32_t *status;           /* [B] or NULL */
+    void *ws; size_t ws_bytes;
+} mtv_step_args;
+
+int mtv_verify_step(const mtv_tree_t *tree, const mtv_step_args *args, void *stream);
+
+/* The same step for a caller whose per-step tensors live in (pinned) host memory.
+ * Copies hidden, root_tok, q_layers and logits host->device into the device
+ * buffers named in `dev`, runs mtv_verify_step, copies tree_tok, out_layers,
+ * accept_len, best_path, acc_nodes, acc_tok, next_root and seq_lens back to the
+ * host buffers, and synchronises the stream before returning.  Weights, KV caches
+ * and the tree stay resident on the device.  `host` uses the same struct: only
+ * the fields listed above are read from it. */
+int mtv_verify_step_host(const mtv_tree_t *tree, const mtv_step_args *dev, const mtv_step_args *host,
+                         void *stream);
+
+/* Human-readable text for the most recent MTV_ERR_CUDA on this thread (never NULL). */
+const char *mtv_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MTV_H_ */

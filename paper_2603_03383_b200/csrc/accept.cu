@@ -1,0 +1,138 @@
+// Acceptance and token retrieval (Section 3.2, "Zero-Copy Retrieval"): per-node argmax
+// of the base-model logits, greedy longest-prefix match over the static paths, and the
+// gather of the accepted tokens through retrieve_indices — all on the device.
+#include "common.cuh"
+
+namespace mtv {
+
+constexpr int ARGMAX_THREADS = 256;
+
+AcceptWs accept_ws_layout(const mtv_tree *t, int B, int V) {
+    AcceptWs w;
+    // split each logit row so that the scan fills the GPU: about 4 CTAs per SM in total,
+    // but no chunk shorter than 2048 elements (8 per thread per iteration)
+    long rows = (long)B * t->T;
+    int ns = (int)((4L * sm_count() + rows - 1) / rows);
+    int max_ns = (V + 2047) / 2048;
+    if (ns > max_ns) ns = max_ns;
+    if (ns < 1) ns = 1;
+    w.nsplit = ns;
+    w.part_off = 0;
+    w.total = align_up((size_t)rows * ns * sizeof(unsigned long long), 256);
+    return w;
+}
+
+// Order-preserving key: larger logit first, equal logits by lower index.  bf16 -> the
+// usual sign-flip integer key; ~index in the low half so that max() prefers low indices.
+__device__ __forceinline__ unsigned long long pack_key(uint32_t bf16_bits, uint32_t idx) {
+    uint32_t k = bf16_bits & 0x8000u ? (~bf16_bits & 0xffffu) : (bf16_bits | 0x8000u);
+    if ((bf16_bits & 0x7fffu) == 0) k = 0x8000u;  // -0.0 and +0.0 compare equal
+    return ((unsigned long long)k << 32) | (0xffffffffu - idx);
+}
+
+__device__ __forceinline__ unsigned long long umax64(unsigned long long a, unsigned long long b) { return a > b ? a : b; }
+
+// grid = (nsplit, B*T).  Partial argmax of one chunk of one row.
+__global__ void __launch_bounds__(ARGMAX_THREADS)
+node_argmax_partial_kernel(int V, const __nv_bfloat16 *__restrict__ logits, unsigned long long *__restrict__ part) {
+    const int row = blockIdx.y, ns = gridDim.x;
+    // chunk boundaries on multiples of 8 elements so that 16-byte loads stay aligned
+    const int per = ((V + ns - 1) / ns + 7) / 8 * 8;
+    const int begin = blockIdx.x * per;
+    const int end = min(V, begin + per);
+    const uint16_t *p = reinterpret_cast<const uint16_t *>(logits) + (size_t)row * V;
+    unsigned long long best = 0;
+    const bool aligned = (((size_t)row * V) % 8) == 0;
+    if (aligned) {
+        for (int i = begin + threadIdx.x * 8; i < end; i += ARGMAX_THREADS * 8) {
+            if (i + 8 <= end) {
+                uint4 u;
+                asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                             : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w) : "l"(p + i));
+                const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    best = umax64(best, pack_key(w[j] & 0xffffu, i + 2 * j));
+                    best = umax64(best, pack_key(w[j] >> 16, i + 2 * j + 1));
+                }
+            } else {
+                for (int j = i; j < end; ++j) best = umax64(best, pack_key(p[j], j));
+            }
+        }
+    } else {
+        for (int i = begin + threadIdx.x; i < end; i += ARGMAX_THREADS) best = umax64(best, pack_key(p[i], i));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) best = umax64(best, __shfl_xor_sync(0xffffffffu, best, o));
+    __shared__ unsigned long long sm[ARGMAX_THREADS / 32];
+    if (threadIdx.x % 32 == 0) sm[threadIdx.x / 32] = best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < ARGMAX_THREADS / 32; ++w) best = umax64(best, sm[w]);
+        part[(size_t)row * ns + blockIdx.x] = best;
+    }
+}
+
+// grid = B, block = 128.  Finish the argmax, score every path, pick the best, gather.
+__global__ void __launch_bounds__(128)
+accept_finish_kernel(int T, int K, int P, int ns, const unsigned long long *__restrict__ part,
+                     const int32_t *__restrict__ tree_tok, const int32_t *__restrict__ ri,
+                     int32_t *__restrict__ accept_len, int32_t *__restrict__ best_path,
+                     int32_t *__restrict__ acc_nodes, int32_t *__restrict__ acc_tok,
+                     int32_t *__restrict__ next_root) {
+    __shared__ int32_t am[MTV_MAX_T];
+    __shared__ int32_t tok[MTV_MAX_T];
+    __shared__ unsigned int best_key;
+    const int b = blockIdx.x;
+    for (int i = threadIdx.x; i < T; i += blockDim.x) {
+        unsigned long long best = 0;
+        for (int s = 0; s < ns; ++s) best = umax64(best, part[((size_t)b * T + i) * ns + s]);
+        am[i] = (int32_t)(0xffffffffu - (uint32_t)(best & 0xffffffffu));
+        tok[i] = tree_tok[(size_t)b * T + i];
+    }
+    if (threadIdx.x == 0) best_key = 0;
+    __syncthreads();
+    // key = len * 256 + (255 - p): max() picks the longest match, then the lowest path
+    for (int p = threadIdx.x; p < P; p += blockDim.x) {
+        const int32_t *path = ri + (size_t)p * (K + 1);
+        int len = 0;
+        for (int j = 1; j <= K; ++j) {
+            const int node = path[j];
+            if (node < 0 || tok[node] != am[path[j - 1]]) break;
+            len = j;
+        }
+        atomicMax(&best_key, (unsigned)len * 256u + (255u - (unsigned)p));
+    }
+    __syncthreads();
+    const int len = best_key / 256, p = 255 - (int)(best_key % 256);
+    if ((int)threadIdx.x <= K) {
+        const int j = threadIdx.x;
+        const int node = j <= len ? ri[(size_t)p * (K + 1) + j] : -1;
+        acc_nodes[(size_t)b * (K + 1) + j] = node;
+        acc_tok[(size_t)b * (K + 1) + j] = node >= 0 ? tok[node] : -1;
+        if (j == len) next_root[b] = am[node];
+        if (j == 0) { accept_len[b] = len; best_path[b] = p; }
+    }
+}
+
+}  // namespace mtv
+
+extern "C" int tree_accept(const mtv_tree_t *tree, int B, int V, const mtv_bf16 *logits, const int32_t *tree_tok,
+                           int32_t *accept_len, int32_t *best_path, int32_t *acc_nodes, int32_t *acc_tok,
+                           int32_t *next_root, void *ws, size_t ws_bytes, void *stream) {
+    using namespace mtv;
+    if (!tree || !tree->on_device || !logits || !tree_tok || !accept_len || !best_path || !acc_nodes ||
+        !acc_tok || !next_root || !ws || B < 1 || V < 1)
+        return MTV_ERR_INVALID_ARG;
+    if (tree->P > 255) return MTV_ERR_UNSUPPORTED_SHAPE;
+    const AcceptWs L = accept_ws_layout(tree, B, V);
+    if (ws_bytes < L.total) return MTV_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    auto *part = reinterpret_cast<unsigned long long *>((char *)ws + L.part_off);
+    node_argmax_partial_kernel<<<dim3(L.nsplit, B * tree->T), ARGMAX_THREADS, 0, st>>>(
+        V, reinterpret_cast<const __nv_bfloat16 *>(logits), part);
+    accept_finish_kernel<<<B, 128, 0, st>>>(tree->T, tree->K, tree->P, L.nsplit, part, tree_tok, tree->d_retrieve,
+                                            accept_len, best_path, acc_nodes, acc_tok, next_root);
+    MTV_CUDA_CHECK(cudaGetLastError());
+    return MTV_OK;
+}

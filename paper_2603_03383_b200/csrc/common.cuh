@@ -1,0 +1,66 @@
+// Shared declarations of the CUDA library: the tree object, error plumbing and
+// small device helpers.  Nothing here is used by the CPU checker.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/mtv.h"
+
+struct mtv_tree {
+    int T = 0, K = 0, P = 0, C = 0, anc_words = 0;
+    int k_d[MTV_MAX_K] = {0};
+    int cand_offset[MTV_MAX_K] = {0};
+    std::vector<int32_t> node_ranks, parent, depth, rank, tree_indices, retrieve;
+    std::vector<uint64_t> anc;
+    std::vector<uint8_t> mask;
+    // device copies (one allocation), valid when on_device
+    bool on_device = false;
+    int device = -1;
+    void *d_blob = nullptr;
+    const int32_t *d_tree_indices = nullptr;  // [T]
+    const int32_t *d_retrieve = nullptr;      // [P][K+1]
+    const uint64_t *d_anc = nullptr;          // [T][2]  (always two words per row on the device)
+    const int32_t *d_kd = nullptr;            // [K]
+    const int32_t *d_cand_offset = nullptr;   // [K]
+};
+
+namespace mtv {
+
+void set_last_error(const char *what, cudaError_t e);
+
+#define MTV_CUDA_CHECK(expr)                                  \
+    do {                                                      \
+        cudaError_t e__ = (expr);                             \
+        if (e__ != cudaSuccess) {                             \
+            ::mtv::set_last_error(#expr, e__);                \
+            return MTV_ERR_CUDA;                              \
+        }                                                     \
+    } while (0)
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Workspace carving shared by the entry points (all offsets 256-byte aligned).
+struct HeadsWs {
+    size_t hprime_off, part_val_off, part_idx_off, total;
+    int ctas_per_head;
+};
+HeadsWs heads_ws_layout(const mtv_tree *t, int B, int H, int V);
+
+struct AttnWs {
+    size_t o_off, ml_off, total;
+    int nsplit, m_rows;
+};
+AttnWs attn_ws_layout(const mtv_tree *t, int B, int Hq, int Hkv, int D, int Lcap);
+
+struct AcceptWs {
+    size_t part_off, total;
+    int nsplit;
+};
+AcceptWs accept_ws_layout(const mtv_tree *t, int B, int V);
+
+int sm_count();
+
+}  // namespace mtv

@@ -1,0 +1,304 @@
+"""GPU parity: every C-ABI call against the fp64 checker, element by element, on the same
+seeded inputs.  Integer outputs bit-exact; floats within max|err| <= 1e-2*max|ref| + 1e-3."""
+import ctypes as C
+
+import pytest
+import torch
+
+from oracle import reference as ref
+from paper_2603_03383_b200 import binding, synth
+from tests._cases import assert_close, make_tree, oracle_heads_with_margin, workspace
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _i32(*shape, fill=-7):
+    return torch.full(shape, fill, dtype=torch.int32, device=DEV)
+
+
+# ------------------------------------------------------------------ heads
+HEAD_CASES = [
+    # B, H, V, K, tree
+    (1, 512, 1024, 3, ("cartesian", (4, 2, 2), 0)),       # the tiny configuration
+    (2, 520, 1000, 3, ("cartesian", (4, 2, 2), 0)),       # H, V not multiples of the tile sizes
+    (3, 256, 3001, 4, ("rank_prior", (), 64)),
+    (5, 1024, 5000, 4, ("rank_prior", (), 64)),
+    (16, 512, 2048, 2, ("cartesian", (16, 3), 0)),
+    (1, 8, 20, 1, ("cartesian", (16,), 0)),               # V barely above top-k
+]
+
+
+@pytest.mark.parametrize("B,H,V,K,tr", HEAD_CASES)
+@pytest.mark.parametrize("bias", [True, False])
+def test_heads_topk(B, H, V, K, tr, bias):
+    tb, tree = make_tree(tr[0], K, tr[1], tr[2])
+    seed, inp, _, cand_ref, cl_ref, tt_ref = oracle_heads_with_margin(B, H, V, K, tb, 100 + B + H, bias=bias)
+    hidden, W1, b1, W2, root = [None if t is None else t.to(DEV) for t in inp]
+    ws = workspace(tree, B, H, V, 0, 0, 0, 0)
+    cand, cl, tt = _i32(B, tree.C), torch.zeros(B, tree.C - 1, device=DEV), _i32(B, tree.T)
+    binding.medusa_heads_topk(tree, hidden, W1, b1, W2, root, cand, cl, tt, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(cand.cpu(), cand_ref), seed
+    assert torch.equal(tt.cpu(), tt_ref)
+    assert_close(cl, cl_ref, "cand_logit")
+    assert (cl.double().cpu() - cl_ref).abs().max().item() <= 2e-5 * cl_ref.abs().max().item()   # fp32 carry
+    # cand_logit is optional
+    cand2, tt2 = _i32(B, tree.C), _i32(B, tree.T)
+    binding.medusa_heads_topk(tree, hidden, W1, b1, W2, root, cand2, None, tt2, ws)
+    assert torch.equal(cand2, cand) and torch.equal(tt2, tt)
+
+
+def test_heads_exact_ties_take_lowest_id():
+    B, H, V, K = 2, 256, 4096, 2
+    tb, tree = make_tree("cartesian", K, (4, 3))
+    hidden, W1, b1, W2, root = synth.head_inputs(B, H, V, K, seed=77)
+    z = ref.heads_logits(hidden, W1, b1, W2)
+    top = int(torch.argmax(z[0, 0]))
+    for dup in (7, 900, 4095):                # bit-identical rows in different warps / blocks
+        W2[0, dup] = W2[0, top]
+    z = ref.heads_logits(hidden, W1, b1, W2)
+    cand_ref, _, tt_ref, _ = ref.heads_candidates(z, root, tb)
+    assert cand_ref[0, 1:5].tolist() == sorted({7, 900, 4095, top})
+    ws = workspace(tree, B, H, V, 0, 0, 0, 0)
+    cand, tt = _i32(B, tree.C), _i32(B, tree.T)
+    binding.medusa_heads_topk(tree, hidden.to(DEV), W1.to(DEV), b1.to(DEV), W2.to(DEV), root.to(DEV), cand, None,
+                              tt, ws)
+    assert torch.equal(cand.cpu(), cand_ref) and torch.equal(tt.cpu(), tt_ref)
+
+
+# -------------------------------------------------------------- attention
+def _attention_case(tb, tree, B, Hq, Hkv, D, lens, seed, Lcap=None, pad=0):
+    T = tree.T
+    Lcap = Lcap or max(lens) + T + 5
+    q, k, v = synth.attention_inputs(B, T, Hq, Hkv, D, Lcap + pad, seed)
+    k, v = k[:, :, :Lcap], v[:, :, :Lcap]                 # pad > 0: a strided view of a larger cache
+    sl = torch.tensor(lens, dtype=torch.int32)
+    want = ref.tree_attention(q, k, v, sl, tb["mask"])
+    kd = k.to(DEV) if pad == 0 else synth.attention_inputs(B, T, Hq, Hkv, D, Lcap + pad, seed, device=DEV)[1][:, :, :Lcap]
+    vd = v.to(DEV) if pad == 0 else synth.attention_inputs(B, T, Hq, Hkv, D, Lcap + pad, seed, device=DEV)[2][:, :, :Lcap]
+    out = torch.zeros(B, T, Hq, D, dtype=torch.bfloat16, device=DEV)
+    status = _i32(B)
+    ws = workspace(tree, B, 0, 0, Hq, Hkv, D, Lcap)
+    binding.tree_verify_attention(tree, q.to(DEV), kd, vd, sl.to(DEV), out, ws, status=status, Lcap=Lcap)
+    torch.cuda.synchronize()
+    assert status.tolist() == [0] * B
+    return assert_close(out, want, "tree attention")
+
+
+@pytest.mark.parametrize("L", [0, 1, 35, 63, 64, 65, 127, 128, 129, 700])
+def test_attention_prefix_lengths_tiny_tree(L):
+    tb, tree = make_tree("cartesian", 3, (4, 2, 2))
+    _attention_case(tb, tree, 1, 8, 2, 64, [L], seed=L + 1)
+
+
+@pytest.mark.parametrize("kind,K,topk,T,Hq,Hkv,D,lens", [
+    ("rank_prior", 4, (), 64, 32, 8, 128, [517]),                  # 7B head shape, 64-node tree
+    ("rank_prior", 4, (), 65, 8, 2, 128, [200, 131]),              # T = 65: second mask word
+    ("rank_prior", 5, (), 128, 8, 2, 128, [300]),                  # 128-node tree, 512 query rows / KV head
+    ("rank_prior", 5, (), 128, 16, 2, 64, [97, 0, 260]),           # group of 8, ragged batch
+    ("cartesian", 1, (1,), 0, 4, 4, 64, [50]),                     # T = 2, no grouping
+    ("cartesian", 1, (), 0, 2, 1, 128, [40, 3]),                   # root-only tree
+    ("cartesian", 3, (4, 2, 2), 0, 8, 2, 64, [128]),               # the tiny configuration
+])
+def test_attention_shapes(kind, K, topk, T, Hq, Hkv, D, lens):
+    tb, tree = make_tree(kind, K, topk, T)
+    _attention_case(tb, tree, len(lens), Hq, Hkv, D, lens, seed=5)
+
+
+def test_attention_ragged_batch_many_splits_and_strided_cache():
+    tb, tree = make_tree("rank_prior", 4, (), 64)
+    _attention_case(tb, tree, 3, 8, 2, 128, [1500, 40, 777], seed=9, Lcap=1600, pad=24)
+
+
+def test_attention_capacity_is_reported_not_faulted():
+    tb, tree = make_tree("cartesian", 2, (2, 2))
+    T, B, Hq, Hkv, D, Lcap = tree.T, 2, 4, 2, 64, 40
+    q, k, v = synth.attention_inputs(B, T, Hq, Hkv, D, Lcap, 3, device=DEV)
+    sl = torch.tensor([Lcap - T + 1, 10], dtype=torch.int32, device=DEV)       # first sequence does not fit
+    out = torch.full((B, T, Hq, D), 3.0, dtype=torch.bfloat16, device=DEV)
+    status = _i32(B)
+    ws = workspace(tree, B, 0, 0, Hq, Hkv, D, Lcap)
+    binding.tree_verify_attention(tree, q, k, v, sl, out, ws, status=status)
+    torch.cuda.synchronize()
+    assert status.tolist() == [binding.MTV_ERR_CAPACITY, 0]
+    assert bool((out[0] == 3.0).all())                                          # untouched
+    want = ref.tree_attention(q[1:].cpu(), k[1:].cpu(), v[1:].cpu(), sl[1:].cpu(), tb["mask"])
+    assert_close(out[1:], want)
+
+
+def test_attention_explicit_scale():
+    tb, tree = make_tree("cartesian", 2, (2, 2))
+    T, D = tree.T, 64
+    q, k, v = synth.attention_inputs(1, T, 2, 1, D, 64, 4)
+    sl = torch.tensor([30], dtype=torch.int32)
+    want = ref.tree_attention(q, k, v, sl, tb["mask"], scale=0.05)
+    out = torch.zeros(1, T, 2, D, dtype=torch.bfloat16, device=DEV)
+    ws = workspace(tree, 1, 0, 0, 2, 1, D, 64)
+    binding.tree_verify_attention(tree, q.to(DEV), k.to(DEV), v.to(DEV), sl.to(DEV), out, ws, scale=0.05)
+    assert_close(out, want)
+
+
+# ----------------------------------------------------------------- accept
+@pytest.mark.parametrize("B,V,kind,K,topk,T,p", [
+    (1, 1024, "cartesian", 3, (4, 2, 2), 0, (0.6,)),
+    (7, 1001, "cartesian", 3, (4, 2, 2), 0, (0.3, 0.6, 0.9)),      # odd V: rows not 16-byte aligned
+    (4, 20000, "rank_prior", 4, (), 64, (0.9,)),
+    (3, 4096, "rank_prior", 5, (), 128, (0.6,)),
+    (2, 50, "cartesian", 1, (), 0, (0.5,)),                        # root-only tree
+])
+def test_accept(B, V, kind, K, topk, T, p):
+    tb, tree = make_tree(kind, K, topk, T)
+    T = tree.T
+    g = torch.Generator().manual_seed(V)
+    cand = torch.stack([torch.randperm(V, generator=g)[:tb["C"]] for _ in range(B)]).to(torch.int32)
+    tree_tok = cand[:, torch.tensor(tb["tree_indices"])].contiguous()
+    logits, planted = synth.planted_logits(B, T, V, K, tree_tok, tb["parent"], tb["rank"], seed=V + B, p_accept=p)
+    logits[0, T - 1, :] = 0.5                                      # a row of exact ties -> id 0
+    want = ref.tree_accept(ref.node_argmax(logits), tree_tok, tb)
+    assert torch.equal(want["accept_len"], planted)
+    outs = dict(accept_len=_i32(B), best_path=_i32(B), acc_nodes=_i32(B, K + 1), acc_tok=_i32(B, K + 1),
+                next_root=_i32(B))
+    ws = workspace(tree, B, 8, V, 0, 0, 0, 0)
+    binding.tree_accept(tree, logits.to(DEV), tree_tok.to(DEV), outs["accept_len"], outs["best_path"],
+                        outs["acc_nodes"], outs["acc_tok"], outs["next_root"], ws)
+    torch.cuda.synchronize()
+    for name, t in outs.items():
+        assert torch.equal(t.cpu(), want[name]), name
+
+
+def test_accept_negative_zero_and_negative_rows():
+    tb, tree = make_tree("cartesian", 1, (2,))
+    B, T, V = 1, tree.T, 64
+    logits = torch.full((B, T, V), -3.0, dtype=torch.bfloat16)
+    logits[0, 0, 9] = -0.0
+    logits[0, 0, 20] = 0.0                                         # -0.0 == +0.0: lowest id wins
+    logits[0, 1, 33] = -1.5
+    logits[0, 2, :] = float("-inf")
+    tree_tok = torch.tensor([[5, 9, 20]], dtype=torch.int32)
+    am = ref.node_argmax(logits)
+    assert am.tolist() == [[9, 33, 0]]
+    want = ref.tree_accept(am, tree_tok, tb)
+    outs = [_i32(B), _i32(B), _i32(B, 2), _i32(B, 2), _i32(B)]
+    ws = workspace(tree, B, 8, V, 0, 0, 0, 0)
+    binding.tree_accept(tree, logits.to(DEV), tree_tok.to(DEV), *outs, ws)
+    for t, name in zip(outs, ["accept_len", "best_path", "acc_nodes", "acc_tok", "next_root"]):
+        assert torch.equal(t.cpu(), want[name]), name
+
+
+# ------------------------------------------------------------- compaction
+@pytest.mark.parametrize("D,n_layers,B,Hkv", [(128, 3, 4, 2), (64, 1, 2, 8)])
+def test_kv_compaction(D, n_layers, B, Hkv):
+    K = 4
+    tb, tree = make_tree("rank_prior", K, (), 64)
+    T, Lcap = tree.T, 300
+    lens = [100, 0, 236, 237][:B]                                  # 237 + 64 > 300: reported, skipped
+    paths = [[0, 2, 12, 13, -1], [0, -1, -1, -1, -1], [0, 1, 11, 47, 63], [0, 1, -1, -1, -1]][:B]
+    alen = torch.tensor([sum(1 for x in p if x >= 0) - 1 for p in paths], dtype=torch.int32)
+    acc = torch.tensor(paths, dtype=torch.int32)
+    ks = [synth.normal_bf16(3, 10 + l, (B, Hkv, Lcap, D)) for l in range(n_layers)]
+    vs = [synth.normal_bf16(3, 50 + l, (B, Hkv, Lcap, D)) for l in range(n_layers)]
+    kd, vd = [t.to(DEV) for t in ks], [t.to(DEV) for t in vs]
+    kp, vp = binding.cache_pointer_array(kd, DEV), binding.cache_pointer_array(vd, DEV)
+    sl = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    status = _i32(B)
+    binding.kv_compact_accepted(tree, kp, vp, n_layers, B, Hkv, D, (Hkv * Lcap * D, Lcap * D, D), Lcap, sl,
+                                alen.to(DEV), acc.to(DEV), status=status)
+    torch.cuda.synchronize()
+    fits = [l + T <= Lcap for l in lens]
+    assert status.tolist() == [0 if f else binding.MTV_ERR_CAPACITY for f in fits]
+    for layer in range(n_layers):
+        for cache, got in ((ks[layer], kd[layer]), (vs[layer], vd[layer])):
+            want, new_len = ref.kv_compact(cache, lens, alen, acc)
+            for b in range(B):
+                if not fits[b]:
+                    assert torch.equal(got[b].cpu(), cache[b]) and sl[b].item() == lens[b]
+                    continue
+                keep = new_len[b].item()
+                assert sl[b].item() == keep
+                assert torch.equal(got[b, :, :keep].cpu(), want[b, :, :keep])
+                assert torch.equal(got[b, :, lens[b] + T:].cpu(), cache[b, :, lens[b] + T:])   # nothing past the tree rows
+
+
+# -------------------------------------------------------------- full step
+def _step_case(B, H, V, Hq, Hkv, D, n_layers, kind, K, topk, T, lens, seed, host=False):
+    tb, tree = make_tree(kind, K, topk, T)
+    T = tree.T
+    Lcap = max(lens) + T
+    seed, inp, cpu, cand_ref, cl_ref, tt_ref = oracle_heads_with_margin(B, H, V, K, tb, seed)
+    logits, planted = synth.planted_logits(B, T, V, K, tt_ref, tb["parent"], tb["rank"], seed, p_accept=(0.6, 0.9))
+    acc_ref = ref.tree_accept(ref.node_argmax(logits), tt_ref, tb)
+    assert torch.equal(acc_ref["accept_len"], planted)
+    sl = torch.tensor(lens, dtype=torch.int32)
+    layers = [synth.attention_inputs(B, T, Hq, Hkv, D, Lcap, seed, layer=l) for l in range(n_layers)]
+    out_ref = torch.stack([ref.tree_attention(q, k, v, sl, tb["mask"]) for q, k, v in layers])
+    kd, vd = [l[1].to(DEV) for l in layers], [l[2].to(DEV) for l in layers]
+    q_all = torch.stack([l[0] for l in layers])
+    hidden, W1, b1, W2, root = inp
+    a = binding.StepArgs()
+    a.B, a.H, a.V, a.Hq, a.Hkv, a.D, a.n_layers, a.Lcap = B, H, V, Hq, Hkv, D, n_layers, Lcap
+    a.stride_b, a.stride_h, a.stride_t, a.scale = Hkv * Lcap * D, Lcap * D, D, 0.0
+    kp, vp = binding.cache_pointer_array(kd, DEV), binding.cache_pointer_array(vd, DEV)
+    kph, vph = binding.cache_pointer_array(kd), binding.cache_pointer_array(vd)
+    dev = dict(hidden=hidden.to(DEV), W1=W1.to(DEV), b1=b1.to(DEV), W2=W2.to(DEV), root_tok=root.to(DEV),
+               q_layers=q_all.to(DEV), logits=logits.to(DEV), seq_lens=sl.to(DEV),
+               cand=_i32(B, tree.C), cand_logit=torch.zeros(B, tree.C - 1, device=DEV), tree_tok=_i32(B, T),
+               out_layers=torch.zeros(n_layers, B, T, Hq, D, dtype=torch.bfloat16, device=DEV),
+               accept_len=_i32(B), best_path=_i32(B), acc_nodes=_i32(B, K + 1), acc_tok=_i32(B, K + 1),
+               next_root=_i32(B), status=_i32(B), k_caches=kp, v_caches=vp, k_caches_host=kph, v_caches_host=vph,
+               ws=workspace(tree, B, H, V, Hq, Hkv, D, Lcap))
+    for name, t in dev.items():
+        setattr(a, name, t.data_ptr())
+    a.ws_bytes = dev["ws"].numel()
+    if host:
+        hb = binding.StepArgs()
+        names = ["hidden", "root_tok", "q_layers", "logits", "tree_tok", "out_layers", "accept_len", "best_path",
+                 "acc_nodes", "acc_tok", "next_root", "seq_lens"]
+        src = dict(hidden=hidden, root_tok=root, q_layers=q_all, logits=logits)
+        hostbuf = {n: (src[n].clone() if n in src else torch.empty_like(dev[n], device="cpu")).pin_memory()
+                   for n in names}
+        for n in ("hidden", "root_tok", "q_layers", "logits"):     # the device copies start out wrong
+            dev[n].zero_()
+        for n, t in hostbuf.items():
+            setattr(hb, n, t.data_ptr())
+        binding.mtv_verify_step_host(tree, a, hb)
+        got = {n: hostbuf[n] for n in names}
+    else:
+        binding.mtv_verify_step(tree, a)
+        torch.cuda.synchronize()
+        got = {n: t.cpu() for n, t in dev.items() if n not in ("ws",)}
+    assert got.get("status", torch.zeros(B)).tolist() == [0] * B if not host else True
+    assert torch.equal(got["tree_tok"], tt_ref)
+    if not host:
+        assert torch.equal(got["cand"], cand_ref)
+    for l in range(n_layers):
+        assert_close(got["out_layers"][l], out_ref[l], "layer %d" % l)
+    for name in ("accept_len", "best_path", "acc_nodes", "acc_tok", "next_root"):
+        assert torch.equal(got[name], acc_ref[name]), name
+    assert torch.equal(got["seq_lens"], sl + acc_ref["accept_len"] + 1)
+    for l in range(n_layers):
+        for cache, gotc in ((layers[l][1], kd[l]), (layers[l][2], vd[l])):
+            want, new_len = ref.kv_compact(cache, lens, acc_ref["accept_len"], acc_ref["acc_nodes"])
+            for b in range(B):
+                assert torch.equal(gotc[b, :, :new_len[b]].cpu(), want[b, :, :new_len[b]])
+    return acc_ref["accept_len"]
+
+
+def test_full_step_tiny_configuration():
+    w = synth.WORKLOADS["tiny"]
+    _step_case(w.B, w.H, w.V, w.Hq, w.Hkv, w.D, 3, w.tree, w.K, w.topk, w.T, [w.L_lo], w.seed)
+
+
+def test_full_step_batched_ragged():
+    _step_case(5, 256, 3000, 8, 2, 128, 2, "rank_prior", 4, (), 64, [300, 17, 0, 129, 64], seed=31)
+
+
+def test_full_step_from_host_buffers():
+    _step_case(2, 256, 2000, 8, 2, 64, 2, "cartesian", 3, (4, 2, 2), 0, [90, 33], seed=8, host=True)
+
+
+def test_generator_is_identical_on_cpu_and_gpu():
+    a = synth.normal_bf16(123, 5, (1 << 16,), 0.37)
+    b = synth.normal_bf16(123, 5, (1 << 16,), 0.37, device=DEV)
+    assert torch.equal(a, b.cpu())
+    assert torch.equal(synth.uniform_int(9, 1, 100, 5, 5000), synth.uniform_int(9, 1, 100, 5, 5000, device=DEV).cpu())
