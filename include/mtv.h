@@ -220,6 +220,29 @@ int mtv_verify_step(const mtv_tree_t *tree, const mtv_step_args *args, void *str
 int mtv_verify_step_host(const mtv_tree_t *tree, const mtv_step_args *dev, const mtv_step_args *host,
                          void *stream);
 
+/* ---------------------------------------------------------------------------
+ * Measurement aid (the paper has no counterpart): per-kernel device timing.
+ * While taps are set for a kernel id, every launch of that kernel by this library is
+ * bracketed by cudaEventRecord(start[i]) / cudaEventRecord(stop[i]) on the launch
+ * stream, i = 0, 1, ... until `capacity` launches have been recorded; later launches
+ * are not recorded.  start/stop: host arrays of cudaEvent_t created by the caller and
+ * kept alive until the taps are cleared (capacity = 0 or NULL arrays clears them).
+ * Not thread-safe; do not use during stream capture.
+ */
+#define MTV_KERNEL_HEADS_RESBLOCK 0
+#define MTV_KERNEL_HEADS_VOCAB_TOPK 1
+#define MTV_KERNEL_HEADS_MERGE 2
+#define MTV_KERNEL_ATTN_PARTIAL 3
+#define MTV_KERNEL_ATTN_COMBINE 4
+#define MTV_KERNEL_ARGMAX_PARTIAL 5
+#define MTV_KERNEL_ACCEPT_FINISH 6
+#define MTV_KERNEL_KV_COMPACT 7
+#define MTV_KERNEL_SEQ_ADVANCE 8
+#define MTV_KERNEL_COUNT 9
+int mtv_set_kernel_taps(int kernel_id, void **start_events, void **stop_events, int capacity);
+/* Number of launches recorded since the taps of kernel_id were set (-1: bad id). */
+int mtv_kernel_taps_used(int kernel_id);
+
 /* Human-readable text for the most recent MTV_ERR_CUDA on this thread (never NULL). */
 const char *mtv_last_error(void);
 

@@ -24,7 +24,8 @@ MAX_K = 8
 
 EXPORTS = ["tree_build_static", "tree_gen_cartesian", "tree_gen_rank_prior", "tree_query", "tree_destroy",
            "mtv_workspace_bytes", "medusa_heads_topk", "tree_verify_attention", "tree_accept",
-           "kv_compact_accepted", "mtv_verify_step", "mtv_verify_step_host", "mtv_last_error"]
+           "kv_compact_accepted", "mtv_verify_step", "mtv_verify_step_host", "mtv_last_error",
+           "mtv_set_kernel_taps", "mtv_kernel_taps_used"]
 
 
 class MtvError(RuntimeError):
@@ -91,6 +92,8 @@ def lib():
         L.mtv_verify_step.argtypes = [vp, C.POINTER(StepArgs), vp]
         L.mtv_verify_step_host.argtypes = [vp, C.POINTER(StepArgs), C.POINTER(StepArgs), vp]
         L.mtv_last_error.restype = C.c_char_p
+        L.mtv_set_kernel_taps.argtypes = [i32, vp, vp, i32]
+        L.mtv_kernel_taps_used.argtypes = [i32]
         _lib = L
     return _lib
 
@@ -225,3 +228,41 @@ def mtv_verify_step(tree, args: StepArgs, stream=None):
 def mtv_verify_step_host(tree, dev: StepArgs, host: StepArgs, stream=None):
     _check(lib().mtv_verify_step_host(tree.handle, C.byref(dev), C.byref(host), _stream(stream)),
            "mtv_verify_step_host")
+
+
+KERNELS = ["heads_resblock", "heads_vocab_topk", "heads_merge", "attn_partial", "attn_combine",
+           "argmax_partial", "accept_finish", "kv_compact", "seq_advance"]
+
+
+class KernelTaps:
+    """Per-kernel device timing through ``mtv_set_kernel_taps`` (CUDA events on the launch stream)."""
+
+    def __init__(self, capacity_per_kernel: int):
+        self.cap = capacity_per_kernel
+        self.ev = {}
+        for kid, name in enumerate(KERNELS):
+            st = [torch.cuda.Event(enable_timing=True) for _ in range(self.cap)]
+            sp = [torch.cuda.Event(enable_timing=True) for _ in range(self.cap)]
+            for e in st + sp:
+                e.record()          # torch creates the CUDA event lazily: force it now
+            a = (C.c_void_p * self.cap)(*[e.cuda_event for e in st])
+            b = (C.c_void_p * self.cap)(*[e.cuda_event for e in sp])
+            self.ev[kid] = (st, sp, a, b)
+
+    def __enter__(self):
+        for kid, (_, _, a, b) in self.ev.items():
+            _check(lib().mtv_set_kernel_taps(kid, a, b, self.cap), "mtv_set_kernel_taps")
+        return self
+
+    def __exit__(self, *exc):
+        self.used = {kid: lib().mtv_kernel_taps_used(kid) for kid in self.ev}
+        for kid in self.ev:
+            lib().mtv_set_kernel_taps(kid, None, None, 0)
+
+    def times_ms(self):
+        """{kernel name: [ms per recorded launch]} — call after a device synchronize."""
+        out = {}
+        for kid, (st, sp, _, _) in self.ev.items():
+            n = self.used[kid]
+            out[KERNELS[kid]] = [st[i].elapsed_time(sp[i]) for i in range(n)]
+        return out

@@ -129,8 +129,12 @@ extern "C" int tree_accept(const mtv_tree_t *tree, int B, int V, const mtv_bf16 
     if (ws_bytes < L.total) return MTV_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     auto *part = reinterpret_cast<unsigned long long *>((char *)ws + L.part_off);
-    node_argmax_partial_kernel<<<dim3(L.nsplit, B * tree->T), ARGMAX_THREADS, 0, st>>>(
-        V, reinterpret_cast<const __nv_bfloat16 *>(logits), part);
+    {
+        TapScope tap(MTV_KERNEL_ARGMAX_PARTIAL, st);
+        node_argmax_partial_kernel<<<dim3(L.nsplit, B * tree->T), ARGMAX_THREADS, 0, st>>>(
+            V, reinterpret_cast<const __nv_bfloat16 *>(logits), part);
+    }
+    TapScope tap(MTV_KERNEL_ACCEPT_FINISH, st);
     accept_finish_kernel<<<B, 128, 0, st>>>(tree->T, tree->K, tree->P, L.nsplit, part, tree_tok, tree->d_retrieve,
                                             accept_len, best_path, acc_nodes, acc_tok, next_root);
     MTV_CUDA_CHECK(cudaGetLastError());

@@ -325,12 +325,15 @@ extern "C" int tree_verify_attention(const mtv_tree_t *tree, int B, int Hq, int 
         MTV_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_partial_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * BN * 128 * 2));
         attr_done = true;
     }
-    if (D == 64) {
-        tree_attn_partial_kernel<64><<<grid, ATT_THREADS, smem, st>>>(p);
-        tree_attn_combine_kernel<64><<<B * tree->T * Hq, 64, 0, st>>>(p);
-    } else {
-        tree_attn_partial_kernel<128><<<grid, ATT_THREADS, smem, st>>>(p);
-        tree_attn_combine_kernel<128><<<B * tree->T * Hq, 128, 0, st>>>(p);
+    {
+        TapScope tap(MTV_KERNEL_ATTN_PARTIAL, st);
+        if (D == 64) tree_attn_partial_kernel<64><<<grid, ATT_THREADS, smem, st>>>(p);
+        else tree_attn_partial_kernel<128><<<grid, ATT_THREADS, smem, st>>>(p);
+    }
+    {
+        TapScope tap(MTV_KERNEL_ATTN_COMBINE, st);
+        if (D == 64) tree_attn_combine_kernel<64><<<B * tree->T * Hq, 64, 0, st>>>(p);
+        else tree_attn_combine_kernel<128><<<B * tree->T * Hq, 128, 0, st>>>(p);
     }
     MTV_CUDA_CHECK(cudaGetLastError());
     return MTV_OK;

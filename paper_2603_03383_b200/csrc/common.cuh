@@ -63,4 +63,22 @@ AcceptWs accept_ws_layout(const mtv_tree *t, int B, int V);
 
 int sm_count();
 
+// Optional per-kernel event taps (see mtv_set_kernel_taps).
+struct Tap {
+    cudaEvent_t *start = nullptr, *stop = nullptr;
+    int cap = 0, n = 0;
+};
+extern Tap g_taps[MTV_KERNEL_COUNT];
+struct TapScope {
+    Tap &t;
+    cudaStream_t st;
+    bool on;
+    TapScope(int id, cudaStream_t s) : t(g_taps[id]), st(s), on(t.start && t.n < t.cap) {
+        if (on) cudaEventRecord(t.start[t.n], st);
+    }
+    ~TapScope() {
+        if (on) cudaEventRecord(t.stop[t.n++], st);
+    }
+};
+
 }  // namespace mtv

@@ -65,10 +65,14 @@ extern "C" int kv_compact_accepted(const mtv_tree_t *tree, int B, int Hkv, int D
     if (stride_t % 8 || stride_h % 8 || stride_b % 8) return MTV_ERR_INVALID_ARG;
     if (B > 65535 || n_layers > 65535) return MTV_ERR_UNSUPPORTED_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
-    kv_compact_kernel<<<dim3(Hkv, B, n_layers), 256, 0, st>>>(
+    {
+        TapScope tap(MTV_KERNEL_KV_COMPACT, st);
+        kv_compact_kernel<<<dim3(Hkv, B, n_layers), 256, 0, st>>>(
         tree->T, tree->K, D, Lcap, reinterpret_cast<__nv_bfloat16 *const *>(k_caches),
         reinterpret_cast<__nv_bfloat16 *const *>(v_caches), stride_b, stride_h, stride_t, seq_lens, accept_len,
-        acc_nodes);
+            acc_nodes);
+    }
+    TapScope tap(MTV_KERNEL_SEQ_ADVANCE, st);
     seq_lens_advance_kernel<<<(B + 127) / 128, 128, 0, st>>>(B, tree->T, Lcap, seq_lens, accept_len, status);
     MTV_CUDA_CHECK(cudaGetLastError());
     return MTV_OK;

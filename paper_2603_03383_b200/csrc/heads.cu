@@ -299,9 +299,15 @@ static int launch_heads(const mtv_tree *t, int B, int H, int V, const __nv_bfloa
     int g1 = (t->K * H + HEADS_WARPS - 1) / HEADS_WARPS;
     const int cap = 4 * sm_count();
     if (g1 > cap) g1 = cap;
-    heads_resblock_kernel<NB><<<dim3(g1, btiles), HEADS_THREADS, sm1, st>>>(B, H, t->K, hidden, W1, b1, hprime);
-    heads_vocab_topk_kernel<NB><<<dim3(L.ctas_per_head, t->K, btiles), HEADS_THREADS, sm2, st>>>(
-        B, H, V, W2, hprime, t->d_kd, pv, pi);
+    {
+        TapScope tap(MTV_KERNEL_HEADS_RESBLOCK, st);
+        heads_resblock_kernel<NB><<<dim3(g1, btiles), HEADS_THREADS, sm1, st>>>(B, H, t->K, hidden, W1, b1, hprime);
+    }
+    {
+        TapScope tap(MTV_KERNEL_HEADS_VOCAB_TOPK, st);
+        heads_vocab_topk_kernel<NB><<<dim3(L.ctas_per_head, t->K, btiles), HEADS_THREADS, sm2, st>>>(
+            B, H, V, W2, hprime, t->d_kd, pv, pi);
+    }
     return MTV_OK;
 }
 
@@ -338,6 +344,7 @@ extern "C" int medusa_heads_topk(const mtv_tree_t *tree, int B, int H, int V,
         MTV_CUDA_CHECK(cudaFuncSetAttribute(heads_merge_expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
         attr_done = true;
     }
+    TapScope tap(MTV_KERNEL_HEADS_MERGE, st);
     heads_merge_expand_kernel<<<B, tree->K * MERGE_GROUP, smm, st>>>(
         B, tree->K, tree->T, tree->C, L.ctas_per_head,
         reinterpret_cast<const float *>((char *)ws + L.part_val_off),

@@ -39,7 +39,22 @@ int sm_count() {
     }
     return n;
 }
+Tap g_taps[MTV_KERNEL_COUNT];
 }  // namespace mtv
+
+extern "C" int mtv_set_kernel_taps(int id, void **start, void **stop, int capacity) {
+    if (id < 0 || id >= MTV_KERNEL_COUNT) return MTV_ERR_INVALID_ARG;
+    mtv::Tap &t = mtv::g_taps[id];
+    const bool on = start && stop && capacity > 0;
+    t.start = on ? reinterpret_cast<cudaEvent_t *>(start) : nullptr;
+    t.stop = on ? reinterpret_cast<cudaEvent_t *>(stop) : nullptr;
+    t.cap = on ? capacity : 0;
+    t.n = 0;
+    return MTV_OK;
+}
+extern "C" int mtv_kernel_taps_used(int id) {
+    return id < 0 || id >= MTV_KERNEL_COUNT ? -1 : mtv::g_taps[id].n;
+}
 
 extern "C" const char *mtv_last_error(void) { return g_err; }
 
