@@ -153,7 +153,7 @@ def build_problem(w, n_layers, device):
     return d
 
 
-LAUNCHES_PER_STEP = lambda n_layers: 3 + 2 * n_layers + 2 + 2
+LAUNCHES_PER_STEP = lambda n_layers: 2 + 2 * n_layers + 2 + 2
 
 
 def run_ours(args):
@@ -278,7 +278,7 @@ def run_ours(args):
                                 "frac_of_8tbs": ach / 8000.0, "avg_call_us": a_ms * 1e3,
                                 "algorithmic_bytes_per_launch": alg["attn_per_layer"]}
     if not args.no_cpu_baseline and world == 1:
-        out["cpu_baseline"] = cpu_baseline(w, P, n_layers, budget_s=20.0)
+        out["cpu_baseline"] = cpu_baseline(w, P, n_layers, budget_s=25.0)
     elif not args.no_cpu_baseline:
         out["cpu_baseline"] = None
     print(json.dumps(out))
@@ -286,69 +286,86 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def _sample_inputs_from_problem(w, P, vocab_rows):
+def _sample_plan(w, T, n_layers, est_full_s, budget_s):
+    """How much of one step the checker runs so that it takes about budget_s seconds."""
+    f = min(1.0, budget_s / max(est_full_s, 1e-9))
+    n_heads = max(1, min(w.K, int(round(w.K * f))))
+    vocab_rows = w.V if n_heads > 1 else min(w.V, max(2048, int(w.V * w.K * f)))
+    layers = max(1, min(n_layers, int(round(n_layers * f))))
+    total_rows = w.B * T * w.Hq
+    attn_rows = total_rows if layers > 1 else min(total_rows, max(8, int(total_rows * n_layers * f)))
+    logit_rows = max(1, min(T, int(round(T * f))))
+    return dict(n_heads=n_heads, vocab_rows=vocab_rows, layers=layers, attn_rows=attn_rows, logit_rows=logit_rows)
+
+
+def _sample_inputs_from_problem(w, P, plan):
     """CPU copies of the slices the checker's sample needs (same values the CUDA arm uses)."""
-    return dict(hidden=P["hidden"].cpu(), W1=P["W1"][:1].cpu(), b1=P["b1"][:1].cpu(),
-                W2=P["W2"][:1, :vocab_rows].cpu(), q=P["q_layers"][0].cpu(), k=P["k_list"][0].cpu(),
-                v=P["v_list"][0].cpu(), logits=P["logits"][:, :1].cpu(), lens=P["lens"],
-                mask=P["tree"].medusa_attn_mask, T=P["tree"].T)
+    nh, vr, nl, nr = plan["n_heads"], plan["vocab_rows"], plan["layers"], plan["logit_rows"]
+    return dict(hidden=P["hidden"].cpu(), W1=P["W1"][:nh].cpu(), b1=P["b1"][:nh].cpu(),
+                W2=P["W2"][:nh, :vr].cpu(), q=[P["q_layers"][l].cpu() for l in range(nl)],
+                k=[P["k_list"][l].cpu() for l in range(nl)], v=[P["v_list"][l].cpu() for l in range(nl)],
+                logits=P["logits"][:, :nr].cpu(), lens=P["lens"], mask=P["tree"].medusa_attn_mask, T=P["tree"].T)
 
 
-def _sample_inputs_on_cpu(w, vocab_rows):
+def _sample_inputs_on_cpu(w, plan):
     """The same slices generated on the host (the generator is counter-based: a prefix of a
     tensor has the same values as the whole tensor's prefix).  No CUDA code involved."""
     import math
+    import torch
     from oracle import tree as otree
     from paper_2603_03383_b200 import synth
+    nh, vr, nl, nr = plan["n_heads"], plan["vocab_rows"], plan["layers"], plan["logit_rows"]
     nodes = otree.cartesian(w.topk) if w.tree == "cartesian" else otree.rank_prior(w.K, w.T, w.R_max)
     tb = otree.tables(nodes, w.K)
     T, seed, Lcap = tb["T"], w.seed, int(w.L_hi) + tb["T"]
-    q, k, v = synth.attention_inputs(w.B, T, w.Hq, w.Hkv, w.D, Lcap, seed, layer=0)
+    qkv = [synth.attention_inputs(w.B, T, w.Hq, w.Hkv, w.D, Lcap, seed, layer=l) for l in range(nl)]
+    W2 = torch.stack([synth.normal_bf16(seed, synth.TID_W2, (h + 1, w.V, w.H), 1.0 / math.sqrt(w.H))[h, :vr]
+                      for h in range(nh)]) if nh > 1 else \
+        synth.normal_bf16(seed, synth.TID_W2, (1, vr, w.H), 1.0 / math.sqrt(w.H))
+    logits = synth.normal_bf16(seed, synth.TID_LOGITS, (w.B, T, w.V))[:, :nr].contiguous() if w.B > 1 else \
+        synth.normal_bf16(seed, synth.TID_LOGITS, (1, nr, w.V))
     return dict(hidden=synth.normal_bf16(seed, synth.TID_HIDDEN, (w.B, w.H)),
-                W1=synth.normal_bf16(seed, synth.TID_W1, (1, w.H, w.H), 1.0 / math.sqrt(w.H)),
-                b1=synth.normal_bf16(seed, synth.TID_B1, (1, w.H), 0.1),
-                W2=synth.normal_bf16(seed, synth.TID_W2, (1, vocab_rows, w.H), 1.0 / math.sqrt(w.H)),
-                q=q, k=k, v=v, logits=synth.normal_bf16(seed, synth.TID_LOGITS, (w.B, 1, w.V)),
+                W1=synth.normal_bf16(seed, synth.TID_W1, (nh, w.H, w.H), 1.0 / math.sqrt(w.H)),
+                b1=synth.normal_bf16(seed, synth.TID_B1, (nh, w.H), 0.1), W2=W2,
+                q=[t[0] for t in qkv], k=[t[1] for t in qkv], v=[t[2] for t in qkv], logits=logits,
                 lens=synth.seq_lens(w), mask=tb["mask"], T=T)
 
 
-def _oracle_step_sample(w, S, n_layers, attn_rows):
-    """Run the checker on a sample; returns (seconds, estimated seconds for a whole step, description)."""
+def _oracle_step_sample(w, S, n_layers, plan):
+    """Run the checker on the planned sample; returns (seconds, estimated seconds for a whole step, description)."""
     from oracle import reference as ref
     T, B = S["T"], w.B
-    vocab_rows = S["W2"].shape[1]
-    rows = [(r % B, (r * 7) % T, (r * 13) % w.Hq) for r in range(attn_rows)]
+    nh, vr, nl, ar, nr = plan["n_heads"], plan["vocab_rows"], plan["layers"], plan["attn_rows"], plan["logit_rows"]
+    total_rows = B * T * w.Hq
+    rows = None if ar >= total_rows else [(r % B, (r * 7) % T, (r * 13) % w.Hq) for r in range(ar)]
     t0 = time.perf_counter()
     ref.heads_logits(S["hidden"], S["W1"], S["b1"], S["W2"])
     t_head = time.perf_counter() - t0
     t0 = time.perf_counter()
-    ref.tree_attention(S["q"], S["k"], S["v"], S["lens"], S["mask"], rows=rows)
+    for l in range(nl):
+        ref.tree_attention(S["q"][l], S["k"][l], S["v"][l], S["lens"], S["mask"], rows=rows)
     t_attn = time.perf_counter() - t0
     t0 = time.perf_counter()
     ref.node_argmax(S["logits"])
     t_arg = time.perf_counter() - t0
-    # scale each part to the whole step (the W1 block is counted once per head, unscaled by the vocabulary)
-    full = (t_head * w.K * (w.V / vocab_rows) + t_attn * n_layers * (B * T * w.Hq / attn_rows) + t_arg * T)
-    desc = ("1 of %d heads on %d of %d vocabulary rows, %d of %d attention rows of 1 of %d layers, argmax of 1 of %d "
-            "logit rows per sequence; times scaled to a whole step" % (w.K, vocab_rows, w.V, attn_rows,
-                                                                     B * T * w.Hq, n_layers, T))
+    full = (t_head * (w.K / nh) * (w.V / vr) + t_attn * (n_layers / nl) * (total_rows / min(ar, total_rows))
+            + t_arg * (T / nr))
+    desc = ("%d of %d heads on %d of %d vocabulary rows, %d of %d attention rows of %d of %d layers, argmax of %d of %d "
+            "logit rows per sequence; each part's time scaled to a whole step" % (
+                nh, w.K, vr, w.V, min(ar, total_rows), total_rows, nl, n_layers, nr, T))
     return t_head + t_attn + t_arg, full, desc
 
 
-def _size_sample(w, T, n_layers, full_estimate_s, budget_s):
-    frac = min(1.0, budget_s / max(full_estimate_s, 1e-9))
-    total_rows = T * w.B * w.Hq
-    attn_rows = min(total_rows, max(8, int(total_rows * frac)))
-    vocab_rows = min(w.V, max(2048, int(w.V * w.K * frac)))
-    return attn_rows, vocab_rows
+_CALIBRATION = dict(n_heads=1, vocab_rows=2048, layers=1, attn_rows=8, logit_rows=1)
 
 
 def cpu_baseline(w, P, n_layers, budget_s):
     cores = os.cpu_count() or 1
     # calibrate on a small sample, then size the real one to the budget
-    _, full, _ = _oracle_step_sample(w, _sample_inputs_from_problem(w, P, min(w.V, 2048)), n_layers, 8)
-    attn_rows, vocab_rows = _size_sample(w, P["tree"].T, n_layers, full, budget_s)
-    s, full, desc = _oracle_step_sample(w, _sample_inputs_from_problem(w, P, vocab_rows), n_layers, attn_rows)
+    cal = dict(_CALIBRATION, vocab_rows=min(w.V, 2048))
+    _, full, _ = _oracle_step_sample(w, _sample_inputs_from_problem(w, P, cal), n_layers, cal)
+    plan = _sample_plan(w, P["tree"].T, n_layers, full, budget_s)
+    s, full, desc = _oracle_step_sample(w, _sample_inputs_from_problem(w, P, plan), n_layers, plan)
     return {"value": 1.0 / full, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
             "sample_seconds": s}
 
@@ -362,16 +379,17 @@ def run_reference(args):
     n_layers = args.layers
     K_steps, W_steps = args.steps, args.warmup
     per_step_budget = min(5.0, 150.0 / max(1, K_steps + W_steps))
-    S = _sample_inputs_on_cpu(w, min(w.V, 2048))
-    _, full, _ = _oracle_step_sample(w, S, n_layers, 8)
-    attn_rows, vocab_rows = _size_sample(w, S["T"], n_layers, full, per_step_budget)
-    S = _sample_inputs_on_cpu(w, vocab_rows)
+    cal = dict(_CALIBRATION, vocab_rows=min(w.V, 2048))
+    S = _sample_inputs_on_cpu(w, cal)
+    _, full, _ = _oracle_step_sample(w, S, n_layers, cal)
+    plan = _sample_plan(w, S["T"], n_layers, full, per_step_budget)
+    S = _sample_inputs_on_cpu(w, plan)
     for _ in range(W_steps):
-        _oracle_step_sample(w, S, n_layers, attn_rows)
+        _oracle_step_sample(w, S, n_layers, plan)
     fulls, desc = [], ""
     t0 = time.perf_counter()
     for _ in range(K_steps):
-        _, full, desc = _oracle_step_sample(w, S, n_layers, attn_rows)
+        _, full, desc = _oracle_step_sample(w, S, n_layers, plan)
         fulls.append(full)
     wall = time.perf_counter() - t0
     full = sum(fulls) / len(fulls)

@@ -243,6 +243,14 @@ int mtv_set_kernel_taps(int kernel_id, void **start_events, void **stop_events, 
 /* Number of launches recorded since the taps of kernel_id were set (-1: bad id). */
 int mtv_kernel_taps_used(int kernel_id);
 
+/* Sticky device-side error word of the device the tree was uploaded to (the paper has
+ * no counterpart).  A kernel whose bounded wait ran out (a copy or a tensor-core
+ * operation that never signalled completion) stores MTV_ERR_TIMEOUT there and unwinds
+ * instead of spinning; the outputs of that call are then undefined.  *code receives
+ * the word (0 = no error since it was last cleared); clear != 0 resets it.  This call
+ * synchronises with the device: use it between steps, not inside one. */
+int mtv_device_error(const mtv_tree_t *tree, int clear, int32_t *code);
+
 /* Human-readable text for the most recent MTV_ERR_CUDA on this thread (never NULL). */
 const char *mtv_last_error(void);
 

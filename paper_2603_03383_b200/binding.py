@@ -25,7 +25,7 @@ MAX_K = 8
 EXPORTS = ["tree_build_static", "tree_gen_cartesian", "tree_gen_rank_prior", "tree_query", "tree_destroy",
            "mtv_workspace_bytes", "medusa_heads_topk", "tree_verify_attention", "tree_accept",
            "kv_compact_accepted", "mtv_verify_step", "mtv_verify_step_host", "mtv_last_error",
-           "mtv_set_kernel_taps", "mtv_kernel_taps_used"]
+           "mtv_set_kernel_taps", "mtv_kernel_taps_used", "mtv_device_error"]
 
 
 class MtvError(RuntimeError):
@@ -94,6 +94,7 @@ def lib():
         L.mtv_last_error.restype = C.c_char_p
         L.mtv_set_kernel_taps.argtypes = [i32, vp, vp, i32]
         L.mtv_kernel_taps_used.argtypes = [i32]
+        L.mtv_device_error.argtypes = [vp, i32, C.POINTER(C.c_int32)]
         _lib = L
     return _lib
 
@@ -167,6 +168,12 @@ class Tree:
 
 def tree_build_static(K, node_ranks, upload=True) -> Tree:
     return Tree(K, node_ranks, upload)
+
+
+def mtv_device_error(tree: Tree, clear: bool = True) -> int:
+    code = C.c_int32(0)
+    _check(lib().mtv_device_error(tree.handle, 1 if clear else 0, C.byref(code)), "mtv_device_error")
+    return code.value
 
 
 def mtv_workspace_bytes(tree: Tree, B, H, V, Hq, Hkv, D, Lcap) -> int:

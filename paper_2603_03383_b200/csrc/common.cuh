@@ -25,6 +25,7 @@ struct mtv_tree {
     const uint64_t *d_anc = nullptr;          // [T][2]  (always two words per row on the device)
     const int32_t *d_kd = nullptr;            // [K]
     const int32_t *d_cand_offset = nullptr;   // [K]
+    int32_t *d_error = nullptr;               // sticky device-side error word (0 = none)
 };
 
 namespace mtv {
@@ -44,8 +45,8 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 
 // Workspace carving shared by the entry points (all offsets 256-byte aligned).
 struct HeadsWs {
-    size_t hprime_off, part_val_off, part_idx_off, total;
-    int ctas_per_head;
+    size_t hprime_off, part_val_off, part_idx_off, counters_off, total;
+    int ctas_per_head, n_counters;
 };
 HeadsWs heads_ws_layout(const mtv_tree *t, int B, int H, int V);
 

@@ -7,6 +7,7 @@
 // with many loads in flight; activations stay in shared memory in fp32 so that no
 // intermediate is rounded.
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace mtv {
 
@@ -14,18 +15,64 @@ constexpr int HEADS_THREADS = 256;
 constexpr int HEADS_WARPS = HEADS_THREADS / 32;
 constexpr int NB_MAX = 4;  // batch rows handled by one pass over the weights
 
+// vocabulary projection: 2 groups of 8 consumer warps + 1 producer warp
+constexpr int VT_GROUP_WARPS = 8;
+constexpr int VT_GROUPS = 2;
+constexpr int VT_CONS_WARPS = VT_GROUP_WARPS * VT_GROUPS;
+constexpr int VT_THREADS = (VT_CONS_WARPS + 1) * 32;
+constexpr int VT_MAX_STAGES = 6;
+constexpr uint32_t VT_SMEM_MAX = 226 * 1024;  // the opt-in limit minus room for static shared memory
+
+// Shared-memory plan of the vocabulary projection for one (NB, H): rows per stage, number
+// of stages, and the byte offsets of every region.
+struct VocabSmem {
+    int rows_per_stage, n_stages, n_it;
+    uint32_t stage_bytes, ring_bytes, xs_off, lists_off, bars_off, total;
+};
+static VocabSmem vocab_smem_plan(int NB, int H, int ctas_per_head) {
+    VocabSmem s;
+    s.n_it = (H / 8 + 31) / 32;                       // 16-byte chunks per lane and row
+    const uint32_t row_bytes = (uint32_t)H * 2;
+    const uint32_t xs_bytes = (uint32_t)NB * s.n_it * 64 * 16;
+    const uint32_t lists_bytes = (uint32_t)VT_CONS_WARPS * NB * MTV_MAX_TOPK * 8;
+    const uint32_t merge_bytes = (uint32_t)ctas_per_head * MTV_MAX_TOPK * 8;   // final merge reuses the ring
+    const uint32_t fixed = xs_bytes + lists_bytes + 256;
+    s.rows_per_stage = 0;
+    for (int rs = VT_GROUP_WARPS; rs >= 1; rs /= 2) {
+        const uint32_t sb = rs * row_bytes;
+        if (fixed + 2 * sb > VT_SMEM_MAX) continue;
+        int n = (int)((VT_SMEM_MAX - fixed) / sb);
+        if (n > VT_MAX_STAGES) n = VT_MAX_STAGES;
+        // keep at least ~96 KB in flight when the rows are long enough
+        s.rows_per_stage = rs; s.n_stages = n; s.stage_bytes = sb;
+        break;
+    }
+    if (s.rows_per_stage == 0) { s.total = 0; return s; }
+    s.ring_bytes = s.n_stages * s.stage_bytes;
+    if (s.ring_bytes < merge_bytes) s.ring_bytes = (merge_bytes + 127) / 128 * 128;
+    s.xs_off = (s.ring_bytes + 127) / 128 * 128;
+    s.lists_off = s.xs_off + xs_bytes;
+    s.bars_off = s.lists_off + lists_bytes;
+    s.total = s.bars_off + 256;
+    if (s.total > VT_SMEM_MAX) s.total = 0;
+    return s;
+}
+
 HeadsWs heads_ws_layout(const mtv_tree *t, int B, int H, int V) {
     HeadsWs w;
-    // CTAs per head for the vocabulary projection: fill the GPU about twice over all heads
-    int per_head = (2 * sm_count() + t->K - 1) / t->K;
-    int max_useful = (V + HEADS_WARPS - 1) / HEADS_WARPS;  // at least one row per warp
+    // one persistent CTA per SM, the SMs divided evenly among the heads
+    int per_head = sm_count() / t->K;
+    const int max_useful = (V + VT_GROUP_WARPS - 1) / VT_GROUP_WARPS;
     if (per_head > max_useful) per_head = max_useful;
     if (per_head < 1) per_head = 1;
     w.ctas_per_head = per_head;
+    const int btiles = (B + NB_MAX - 1) / NB_MAX;
     size_t off = 0;
     w.hprime_off = off;   off = align_up(off + (size_t)t->K * B * H * sizeof(float), 256);
     w.part_val_off = off; off = align_up(off + (size_t)t->K * B * per_head * MTV_MAX_TOPK * sizeof(float), 256);
     w.part_idx_off = off; off = align_up(off + (size_t)t->K * B * per_head * MTV_MAX_TOPK * sizeof(int32_t), 256);
+    w.counters_off = off; off = align_up(off + (size_t)(t->K + 1) * btiles * sizeof(int32_t), 256);
+    w.n_counters = (t->K + 1) * btiles;
     w.total = off;
     return w;
 }
@@ -65,9 +112,12 @@ template <int NB>
 __global__ void __launch_bounds__(HEADS_THREADS)
 heads_resblock_kernel(int B, int H, int K, const __nv_bfloat16 *__restrict__ hidden,
                       const __nv_bfloat16 *__restrict__ W1, const __nv_bfloat16 *__restrict__ b1,
-                      float *__restrict__ hprime) {
+                      float *__restrict__ hprime, int32_t *__restrict__ counters, int n_counters) {
     extern __shared__ float sh[];  // [NB][H]
     const int b0 = blockIdx.y * NB;
+    // tickets of the vocabulary kernel (the next launch on the stream) start at zero
+    if (blockIdx.x == 0 && blockIdx.y == 0)
+        for (int i = threadIdx.x; i < n_counters; i += HEADS_THREADS) counters[i] = 0;
     for (int i = threadIdx.x; i < NB * H; i += HEADS_THREADS) {
         int b = b0 + i / H;
         sh[i] = b < B ? __bfloat162float(hidden[(size_t)b * H + i % H]) : 0.f;
@@ -107,206 +157,300 @@ heads_resblock_kernel(int B, int H, int K, const __nv_bfloat16 *__restrict__ hid
 }
 
 // ---------------------------------------------------------------------------
-// Vocabulary projection with fused partial top-k.
-// grid = (ctas_per_head, K, ceil(B/NB)).  A CTA owns a contiguous slab of vocabulary
-// rows of one head; each warp walks its rows two at a time, keeps the dot products of
-// NB batch rows in registers and inserts a logit into its private sorted list only
-// when it beats the list's last entry.  At the end the warps' lists are merged and
-// the CTA's best kd entries per batch row go to the workspace.
-template <int NB>
-__global__ void __launch_bounds__(HEADS_THREADS)
-heads_vocab_topk_kernel(int B, int H, int V, const __nv_bfloat16 *__restrict__ W2,
-                        const float *__restrict__ hprime, const int32_t *__restrict__ kd_arr,
-                        float *__restrict__ part_val, int32_t *__restrict__ part_idx) {
-    extern __shared__ float sh[];                   // [NB][H] then the lists
-    float *xs = sh;
-    float *lval = sh + (size_t)NB * H;              // [WARPS][NB][16]
-    int32_t *lidx = reinterpret_cast<int32_t *>(lval + HEADS_WARPS * NB * MTV_MAX_TOPK);
-    const int k = blockIdx.y, b0 = blockIdx.z * NB;
-    const int kd = kd_arr[k];
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    const int per = gridDim.x;
-    if (kd == 0) return;
+// Vocabulary projection with fused top-k, merge and tree expansion.
+//
+// grid = (ctas_per_head, K, ceil(B/NB)): one persistent CTA per SM, each owning a
+// contiguous slab of one head's vocabulary rows.  A producer warp streams the slab
+// through a ring of shared-memory stages with bulk (TMA) copies, one copy per weight
+// row, completion counted on an mbarrier per stage, so that the bytes in flight per SM
+// do not depend on how many registers the consumers have.  Two groups of eight consumer
+// warps take alternate stages; a warp computes the dot products of one weight row with
+// NB activation rows (fp32 activations in shared memory, laid out so that a warp's
+// 16-byte reads are conflict-free) and inserts a logit into its private sorted list only
+// when it beats the list's last entry.  Afterwards the warps' lists are merged per CTA;
+// the last CTA of a head (atomic ticket, no waiting) merges the CTAs' lists into the
+// candidate buffer, and the last head to finish expands the candidates into tree tokens.
+struct VocabParams {
+    int B, H, V, K, T, C;
+    const __nv_bfloat16 *W2;
+    const float *hprime;
+    const int32_t *kd_arr, *off_arr, *tree_indices, *root_tok;
+    float *part_val;
+    int32_t *part_idx;
+    int32_t *counters;   // [btiles][K + 1], zeroed by the residual-block kernel
+    int32_t *cand;
+    float *cand_logit;
+    int32_t *tree_tok;
+    int32_t *dev_error;
+    int rows_per_stage, n_stages, n_it;
+    uint32_t stage_bytes, xs_off, lists_off, bars_off;
+};
 
-    for (int i = threadIdx.x; i < NB * H; i += HEADS_THREADS) {
-        int b = b0 + i / H;
-        xs[i] = b < B ? hprime[((size_t)k * B + b) * H + i % H] : 0.f;
+template <int NB>
+__global__ void __launch_bounds__(VT_THREADS, 1)
+heads_vocab_topk_kernel(const VocabParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    float4 *xs4 = reinterpret_cast<float4 *>(smem + p.xs_off);            // [NB][n_it][2][32]
+    float *lval = reinterpret_cast<float *>(smem + p.lists_off);          // [CONS_WARPS][NB][16]
+    int32_t *lidx = reinterpret_cast<int32_t *>(lval + VT_CONS_WARPS * NB * MTV_MAX_TOPK);
+    const uint32_t bars = ptx::smem_u32(smem + p.bars_off);               // full[n_stages], empty[n_stages]
+    __shared__ int s_flag;
+    __shared__ int s_abort;
+
+    const int k = blockIdx.y, bz = blockIdx.z, b0 = bz * NB;
+    const int per = gridDim.x;
+    const int kd = p.kd_arr[k];
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int H = p.H, RS = p.rows_per_stage, NST = p.n_stages;
+    const uint32_t row_bytes = (uint32_t)H * 2;
+    const int n_chunk16 = H / 8;
+
+    // activations: chunk c = it*32 + lane of row b lives at xs4[((b*n_it + it)*2 + half)*32 + lane]
+    for (int i = threadIdx.x; i < NB * p.n_it * 64; i += VT_THREADS) {
+        const int ln = i % 32, half = (i / 32) % 2, it = (i / 64) % p.n_it, b = i / (64 * p.n_it);
+        const int c = it * 32 + ln;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c < n_chunk16 && b0 + b < p.B)
+            v = *reinterpret_cast<const float4 *>(p.hprime + ((size_t)k * p.B + b0 + b) * H + c * 8 + half * 4);
+        xs4[i] = v;
     }
-    for (int i = threadIdx.x; i < HEADS_WARPS * NB * MTV_MAX_TOPK; i += HEADS_THREADS) {
+    for (int i = threadIdx.x; i < VT_CONS_WARPS * NB * MTV_MAX_TOPK; i += VT_THREADS) {
         lval[i] = -INFINITY;
         lidx[i] = 0x7fffffff;
+    }
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NST; ++s) {
+            ptx::mbar_init(bars + s * 8, 1);                               // full: the producer's expect_tx arrival
+            ptx::mbar_init(bars + (NST + s) * 8, VT_GROUP_WARPS);          // empty: one arrival per consumer warp
+        }
+        ptx::fence_mbar_init();
+        s_abort = 0;
     }
     __syncthreads();
 
     // slab of this CTA
-    const int rows_per = (V + per - 1) / per;
-    const int v_begin = blockIdx.x * rows_per;
-    const int v_end = min(V, v_begin + rows_per);
-    float *my_val = lval + (warp * NB) * MTV_MAX_TOPK;
-    int32_t *my_idx = lidx + (warp * NB) * MTV_MAX_TOPK;
-    float thr_v[NB];
-    int thr_i[NB];
-#pragma unroll
-    for (int b = 0; b < NB; ++b) { thr_v[b] = -INFINITY; thr_i[b] = 0x7fffffff; }
+    const int rows_per = (p.V + per - 1) / per;
+    const int v_begin = min(p.V, (int)blockIdx.x * rows_per);
+    const int v_end = kd > 0 ? min(p.V, v_begin + rows_per) : v_begin;
+    const int n_chunks = (v_end - v_begin + RS - 1) / RS;
+    const __nv_bfloat16 *Wk = p.W2 + (size_t)k * p.V * H;
+    const uint32_t ring = ptx::smem_u32(smem);
+    volatile int *abort_flag = &s_abort;
 
-    const __nv_bfloat16 *Wk = W2 + (size_t)k * V * H;
-    constexpr int R = 2;  // rows per warp iteration
-    for (int v0 = v_begin + warp * R; v0 < v_end; v0 += HEADS_WARPS * R) {
-        float acc[R][NB];
-#pragma unroll
-        for (int r = 0; r < R; ++r)
-#pragma unroll
-            for (int b = 0; b < NB; ++b) acc[r][b] = 0.f;
-        const bool has1 = v0 + 1 < v_end;
-        const __nv_bfloat16 *w0 = Wk + (size_t)v0 * H;
-        const __nv_bfloat16 *w1 = has1 ? w0 + H : w0;
-#pragma unroll 2
-        for (int h0 = lane * 8; h0 < H; h0 += 256) {
-            float wf[R][8];
-            const uint4 u0 = ld_stream(w0 + h0);
-            const uint4 u1 = ld_stream(w1 + h0);
-            bf16x8_to_float(u0, wf[0]);
-            bf16x8_to_float(u1, wf[1]);
-#pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                const float4 x0 = *reinterpret_cast<const float4 *>(xs + b * H + h0);
-                const float4 x1 = *reinterpret_cast<const float4 *>(xs + b * H + h0 + 4);
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    float a = acc[r][b];
-                    a = fmaf(wf[r][0], x0.x, a); a = fmaf(wf[r][1], x0.y, a);
-                    a = fmaf(wf[r][2], x0.z, a); a = fmaf(wf[r][3], x0.w, a);
-                    a = fmaf(wf[r][4], x1.x, a); a = fmaf(wf[r][5], x1.y, a);
-                    a = fmaf(wf[r][6], x1.z, a); a = fmaf(wf[r][7], x1.w, a);
-                    acc[r][b] = a;
-                }
-            }
+    if (warp == VT_CONS_WARPS) {
+        // ---- producer
+        for (int t = 0; t < n_chunks && !*abort_flag; ++t) {
+            const int s = t % NST, use = t / NST;
+            if (use > 0 && !ptx::mbar_wait(bars + (NST + s) * 8, (use - 1) & 1)) { *abort_flag = 1; break; }
+            const int v0 = v_begin + t * RS;
+            const int rows = min(RS, v_end - v0);
+            if (lane == 0) ptx::mbar_arrive_expect_tx(bars + s * 8, rows * row_bytes);
+            __syncwarp();
+            if (lane < rows)
+                ptx::bulk_g2s(ring + s * p.stage_bytes + lane * row_bytes, Wk + (size_t)(v0 + lane) * H, row_bytes,
+                              bars + s * 8);
         }
+    } else {
+        // ---- consumers
+        const int group = warp / VT_GROUP_WARPS, wr = warp % VT_GROUP_WARPS;
+        float *my_val = lval + (warp * NB) * MTV_MAX_TOPK;
+        int32_t *my_idx = lidx + (warp * NB) * MTV_MAX_TOPK;
+        float thr_v[NB];
+        int thr_i[NB];
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            if (r == 1 && !has1) break;
-            const int v = v0 + r;
+        for (int b = 0; b < NB; ++b) { thr_v[b] = -INFINITY; thr_i[b] = 0x7fffffff; }
+        for (int t = group; t < n_chunks; t += VT_GROUPS) {
+            const int s = t % NST, use = t / NST;
+            if (*abort_flag) break;
+            // The two groups take turns on a stage when n_stages is odd.  A parity wait cannot
+            // tell phase `use` from phase `use - 2`, so first make sure that the stage's previous
+            // use was released (by whichever group had it): after that its full barrier is in
+            // phase `use` and the wait below cannot be satisfied by an older phase.
+            if (use > 0 && !ptx::mbar_wait(bars + (NST + s) * 8, (use - 1) & 1)) { *abort_flag = 1; break; }
+            if (!ptx::mbar_wait(bars + s * 8, use & 1)) { *abort_flag = 1; break; }
+            const int v0 = v_begin + t * RS;
+            const int rows = min(RS, v_end - v0);
+            float acc[NB];
 #pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                const float z = warp_sum(acc[r][b]);  // identical in every lane
-                if (cand_before(z, v, thr_v[b], thr_i[b])) {
-                    if (lane == 0) {
-                        // insertion into the sorted list of kd entries
-                        int pos = kd - 1;
-                        while (pos > 0 && cand_before(z, v, my_val[b * MTV_MAX_TOPK + pos - 1],
-                                                      my_idx[b * MTV_MAX_TOPK + pos - 1])) {
-                            my_val[b * MTV_MAX_TOPK + pos] = my_val[b * MTV_MAX_TOPK + pos - 1];
-                            my_idx[b * MTV_MAX_TOPK + pos] = my_idx[b * MTV_MAX_TOPK + pos - 1];
-                            --pos;
+            for (int b = 0; b < NB; ++b) acc[b] = 0.f;
+            if (wr < rows) {
+                const uint4 *wrow = reinterpret_cast<const uint4 *>(smem + s * p.stage_bytes + wr * row_bytes);
+                float acc2[NB];
+#pragma unroll
+                for (int b = 0; b < NB; ++b) acc2[b] = 0.f;
+#pragma unroll 4
+                for (int it = 0; it < p.n_it; ++it) {
+                    const int c = it * 32 + lane;
+                    if (c < n_chunk16) {
+                        float wf[8];
+                        bf16x8_to_float(wrow[c], wf);
+#pragma unroll
+                        for (int b = 0; b < NB; ++b) {
+                            const float4 x0 = xs4[((b * p.n_it + it) * 2) * 32 + lane];
+                            const float4 x1 = xs4[((b * p.n_it + it) * 2 + 1) * 32 + lane];
+                            float a = acc[b], a2 = acc2[b];
+                            a = fmaf(wf[0], x0.x, a); a2 = fmaf(wf[1], x0.y, a2);
+                            a = fmaf(wf[2], x0.z, a); a2 = fmaf(wf[3], x0.w, a2);
+                            a = fmaf(wf[4], x1.x, a); a2 = fmaf(wf[5], x1.y, a2);
+                            a = fmaf(wf[6], x1.z, a); a2 = fmaf(wf[7], x1.w, a2);
+                            acc[b] = a; acc2[b] = a2;
                         }
-                        my_val[b * MTV_MAX_TOPK + pos] = z;
-                        my_idx[b * MTV_MAX_TOPK + pos] = v;
                     }
-                    __syncwarp();
-                    thr_v[b] = my_val[b * MTV_MAX_TOPK + kd - 1];
-                    thr_i[b] = my_idx[b * MTV_MAX_TOPK + kd - 1];
+                }
+#pragma unroll
+                for (int b = 0; b < NB; ++b) acc[b] += acc2[b];
+            }
+            float z[NB];
+#pragma unroll
+            for (int b = 0; b < NB; ++b) z[b] = warp_sum(acc[b]);     // identical in every lane
+            // every lane's reads of the stage are complete (their values fed the sums): release it
+            if (lane == 0) ptx::mbar_arrive(bars + (NST + s) * 8);
+            if (wr < rows) {
+                const int v = v0 + wr;
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    if (cand_before(z[b], v, thr_v[b], thr_i[b])) {
+                        if (lane == 0) {
+                            // insertion into the sorted list of kd entries
+                            int pos = kd - 1;
+                            while (pos > 0 && cand_before(z[b], v, my_val[b * MTV_MAX_TOPK + pos - 1],
+                                                          my_idx[b * MTV_MAX_TOPK + pos - 1])) {
+                                my_val[b * MTV_MAX_TOPK + pos] = my_val[b * MTV_MAX_TOPK + pos - 1];
+                                my_idx[b * MTV_MAX_TOPK + pos] = my_idx[b * MTV_MAX_TOPK + pos - 1];
+                                --pos;
+                            }
+                            my_val[b * MTV_MAX_TOPK + pos] = z[b];
+                            my_idx[b * MTV_MAX_TOPK + pos] = v;
+                        }
+                        __syncwarp();
+                        thr_v[b] = my_val[b * MTV_MAX_TOPK + kd - 1];
+                        thr_i[b] = my_idx[b * MTV_MAX_TOPK + kd - 1];
+                    }
                 }
             }
         }
     }
     __syncthreads();
-    // merge the warps' lists: rank each entry among all HEADS_WARPS*kd entries of its batch row
-    for (int e = threadIdx.x; e < NB * HEADS_WARPS * MTV_MAX_TOPK; e += HEADS_THREADS) {
-        const int b = e / (HEADS_WARPS * MTV_MAX_TOPK);
-        const int w = (e / MTV_MAX_TOPK) % HEADS_WARPS, s = e % MTV_MAX_TOPK;
-        if (s >= kd || b0 + b >= B) continue;
-        const float z = lval[(w * NB + b) * MTV_MAX_TOPK + s];
-        const int id = lidx[(w * NB + b) * MTV_MAX_TOPK + s];
+    if (s_abort) {
+        // A wait ran out.  Raise the sticky error; the producer gives its copies in flight one
+        // more bounded chance to land before the CTA (and its shared memory) goes away.
+        if (threadIdx.x == 0) atomicExch(p.dev_error, MTV_ERR_TIMEOUT);
+        if (warp == VT_CONS_WARPS && lane == 0)
+            for (int s = 0; s < NST; ++s) { ptx::mbar_wait(bars + s * 8, 0); ptx::mbar_wait(bars + s * 8, 1); }
+        return;
+    }
+
+    // ---- merge the warps' lists: rank each entry among all CONS_WARPS*kd entries of its batch row
+    for (int e = threadIdx.x; e < NB * VT_CONS_WARPS * MTV_MAX_TOPK; e += VT_THREADS) {
+        const int b = e / (VT_CONS_WARPS * MTV_MAX_TOPK);
+        const int w = (e / MTV_MAX_TOPK) % VT_CONS_WARPS, sl = e % MTV_MAX_TOPK;
+        if (sl >= kd || b0 + b >= p.B) continue;
+        const float zz = lval[(w * NB + b) * MTV_MAX_TOPK + sl];
+        const int id = lidx[(w * NB + b) * MTV_MAX_TOPK + sl];
         int rank = 0;
-        for (int w2 = 0; w2 < HEADS_WARPS; ++w2)
+        for (int w2 = 0; w2 < VT_CONS_WARPS; ++w2)
             for (int s2 = 0; s2 < kd; ++s2) {
                 const float z2 = lval[(w2 * NB + b) * MTV_MAX_TOPK + s2];
                 const int id2 = lidx[(w2 * NB + b) * MTV_MAX_TOPK + s2];
-                // entries with the sentinel id are all "equal"; order them by position
-                if (cand_before(z2, id2, z, id) || (z2 == z && id2 == id && (w2 * MTV_MAX_TOPK + s2) < (w * MTV_MAX_TOPK + s)))
+                // unused slots all carry the same sentinel: order them by position
+                if (cand_before(z2, id2, zz, id) || (z2 == zz && id2 == id && (w2 * MTV_MAX_TOPK + s2) < (w * MTV_MAX_TOPK + sl)))
                     ++rank;
             }
         if (rank < kd) {
-            const size_t o = (((size_t)k * B + b0 + b) * per + blockIdx.x) * MTV_MAX_TOPK + rank;
-            part_val[o] = z;
-            part_idx[o] = id;
+            const size_t o = (((size_t)k * p.B + b0 + b) * per + blockIdx.x) * MTV_MAX_TOPK + rank;
+            p.part_val[o] = zz;
+            p.part_idx[o] = id;
         }
     }
-}
-
-// ---------------------------------------------------------------------------
-// Final merge + expansion.  grid = B, block = K * 128 threads: thread group d merges
-// head d's per-CTA lists into cand[b][offset_d ..], then the block gathers
-// tree_tok[b][i] = cand[b][tree_indices[i]].
-constexpr int MERGE_GROUP = 128;
-__global__ void heads_merge_expand_kernel(int B, int K, int T, int C, int per,
-                                          const float *__restrict__ part_val,
-                                          const int32_t *__restrict__ part_idx,
-                                          const int32_t *__restrict__ kd_arr,
-                                          const int32_t *__restrict__ off_arr,
-                                          const int32_t *__restrict__ tree_indices,
-                                          const int32_t *__restrict__ root_tok,
-                                          int32_t *__restrict__ cand, float *__restrict__ cand_logit,
-                                          int32_t *__restrict__ tree_tok) {
-    extern __shared__ float sh[];  // per group: per*16 values, per*16 ids
-    const int b = blockIdx.x;
-    const int d = threadIdx.x / MERGE_GROUP, t = threadIdx.x % MERGE_GROUP;
-    const int kd = kd_arr[d], off = off_arr[d];
-    const int n = per * kd;
-    float *val = sh + (size_t)d * per * MTV_MAX_TOPK * 2;
-    int32_t *idx = reinterpret_cast<int32_t *>(val + per * MTV_MAX_TOPK);
-    for (int e = t; e < n; e += MERGE_GROUP) {
-        const size_t o = (((size_t)d * B + b) * per + e / kd) * MTV_MAX_TOPK + e % kd;
-        val[e] = part_val[o];
-        idx[e] = part_idx[o];
-    }
+    // ---- last CTA of this head merges the CTAs' lists (ticket: nobody waits)
+    int32_t *counters = p.counters + (size_t)bz * (p.K + 1);
+    __threadfence();
     __syncthreads();
-    for (int e = t; e < n; e += MERGE_GROUP) {
-        const float z = val[e];
-        const int id = idx[e];
-        int rank = 0;
-        for (int e2 = 0; e2 < n && rank < kd; ++e2)
-            if (cand_before(val[e2], idx[e2], z, id) || (val[e2] == z && idx[e2] == id && e2 < e)) ++rank;
-        if (rank < kd) {
-            cand[(size_t)b * C + off + rank] = id;
-            if (cand_logit) cand_logit[(size_t)b * (C - 1) + off - 1 + rank] = z;
+    if (threadIdx.x == 0) s_flag = atomicAdd(&counters[k], 1) == per - 1;
+    __syncthreads();
+    if (!s_flag) return;
+    __threadfence();
+    {
+        float *mval = reinterpret_cast<float *>(smem);                     // the ring is idle now
+        int32_t *midx = reinterpret_cast<int32_t *>(mval + per * MTV_MAX_TOPK);
+        const int n = per * kd, off = p.off_arr[k];
+        for (int b = 0; b < NB && b0 + b < p.B; ++b) {
+            __syncthreads();
+            for (int e = threadIdx.x; e < n; e += VT_THREADS) {
+                const size_t o = (((size_t)k * p.B + b0 + b) * per + e / kd) * MTV_MAX_TOPK + e % kd;
+                mval[e] = __ldcg(p.part_val + o);
+                midx[e] = __ldcg(p.part_idx + o);
+            }
+            __syncthreads();
+            for (int e = threadIdx.x; e < n; e += VT_THREADS) {
+                const float zz = mval[e];
+                const int id = midx[e];
+                int rank = 0;
+                for (int e2 = 0; e2 < n && rank < kd; ++e2)
+                    if (cand_before(mval[e2], midx[e2], zz, id) || (mval[e2] == zz && midx[e2] == id && e2 < e)) ++rank;
+                if (rank < kd) {
+                    p.cand[(size_t)(b0 + b) * p.C + off + rank] = id;
+                    if (p.cand_logit) p.cand_logit[(size_t)(b0 + b) * (p.C - 1) + off - 1 + rank] = zz;
+                }
+            }
         }
     }
-    if (threadIdx.x == 0) cand[(size_t)b * C] = root_tok[b];
-    __threadfence_block();
+    // ---- last head of this batch tile expands the candidates into the tree tokens
+    __threadfence();
     __syncthreads();
-    for (int i = threadIdx.x; i < T; i += blockDim.x)
-        tree_tok[(size_t)b * T + i] = cand[(size_t)b * C + tree_indices[i]];
+    if (threadIdx.x == 0) s_flag = atomicAdd(&counters[p.K], 1) == p.K - 1;
+    __syncthreads();
+    if (!s_flag) return;
+    __threadfence();
+    for (int e = threadIdx.x; e < NB * p.T; e += VT_THREADS) {
+        const int b = b0 + e / p.T, i = e % p.T;
+        if (b >= p.B) break;
+        const int slot = p.tree_indices[i];
+        const int32_t root = p.root_tok[b];
+        if (i == 0) p.cand[(size_t)b * p.C] = root;
+        p.tree_tok[(size_t)b * p.T + i] = slot == 0 ? root : __ldcg(p.cand + (size_t)b * p.C + slot);
+    }
 }
 
 template <int NB>
 static int launch_heads(const mtv_tree *t, int B, int H, int V, const __nv_bfloat16 *hidden,
                         const __nv_bfloat16 *W1, const __nv_bfloat16 *b1, const __nv_bfloat16 *W2,
+                        const int32_t *root_tok, int32_t *cand, float *cand_logit, int32_t *tree_tok,
                         const HeadsWs &L, char *ws, cudaStream_t st) {
     float *hprime = reinterpret_cast<float *>(ws + L.hprime_off);
-    float *pv = reinterpret_cast<float *>(ws + L.part_val_off);
-    int32_t *pi = reinterpret_cast<int32_t *>(ws + L.part_idx_off);
     const int btiles = (B + NB - 1) / NB;
     const size_t sm1 = (size_t)NB * H * sizeof(float);
-    const size_t sm2 = sm1 + (size_t)HEADS_WARPS * NB * MTV_MAX_TOPK * 8;
-    if (sm2 > 227 * 1024) return MTV_ERR_UNSUPPORTED_SHAPE;
+    const VocabSmem S = vocab_smem_plan(NB, H, L.ctas_per_head);
+    if (sm1 > VT_SMEM_MAX || S.total == 0) return MTV_ERR_UNSUPPORTED_SHAPE;
     static bool attr_done = false;
     if (!attr_done) {
-        MTV_CUDA_CHECK(cudaFuncSetAttribute(heads_resblock_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        MTV_CUDA_CHECK(cudaFuncSetAttribute(heads_vocab_topk_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        MTV_CUDA_CHECK(cudaFuncSetAttribute(heads_resblock_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, VT_SMEM_MAX));
+        MTV_CUDA_CHECK(cudaFuncSetAttribute(heads_vocab_topk_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, VT_SMEM_MAX));
         attr_done = true;
     }
     int g1 = (t->K * H + HEADS_WARPS - 1) / HEADS_WARPS;
     const int cap = 4 * sm_count();
     if (g1 > cap) g1 = cap;
+    int32_t *counters = reinterpret_cast<int32_t *>(ws + L.counters_off);
     {
         TapScope tap(MTV_KERNEL_HEADS_RESBLOCK, st);
-        heads_resblock_kernel<NB><<<dim3(g1, btiles), HEADS_THREADS, sm1, st>>>(B, H, t->K, hidden, W1, b1, hprime);
+        heads_resblock_kernel<NB><<<dim3(g1, btiles), HEADS_THREADS, sm1, st>>>(B, H, t->K, hidden, W1, b1, hprime,
+                                                                               counters, L.n_counters);
     }
+    VocabParams p;
+    p.B = B; p.H = H; p.V = V; p.K = t->K; p.T = t->T; p.C = t->C;
+    p.W2 = W2; p.hprime = hprime;
+    p.kd_arr = t->d_kd; p.off_arr = t->d_cand_offset; p.tree_indices = t->d_tree_indices; p.root_tok = root_tok;
+    p.part_val = reinterpret_cast<float *>(ws + L.part_val_off);
+    p.part_idx = reinterpret_cast<int32_t *>(ws + L.part_idx_off);
+    p.counters = counters;
+    p.cand = cand; p.cand_logit = cand_logit; p.tree_tok = tree_tok;
+    p.dev_error = t->d_error;
+    p.rows_per_stage = S.rows_per_stage; p.n_stages = S.n_stages; p.n_it = S.n_it;
+    p.stage_bytes = S.stage_bytes; p.xs_off = S.xs_off; p.lists_off = S.lists_off; p.bars_off = S.bars_off;
     {
         TapScope tap(MTV_KERNEL_HEADS_VOCAB_TOPK, st);
-        heads_vocab_topk_kernel<NB><<<dim3(L.ctas_per_head, t->K, btiles), HEADS_THREADS, sm2, st>>>(
-            B, H, V, W2, hprime, t->d_kd, pv, pi);
+        heads_vocab_topk_kernel<NB><<<dim3(L.ctas_per_head, t->K, btiles), VT_THREADS, S.total, st>>>(p);
     }
     return MTV_OK;
 }
@@ -323,6 +467,7 @@ extern "C" int medusa_heads_topk(const mtv_tree_t *tree, int B, int H, int V,
         return MTV_ERR_INVALID_ARG;
     if (B < 1 || H < 8 || V < 1) return MTV_ERR_INVALID_ARG;
     if (B > 16 || H % 8 != 0) return MTV_ERR_UNSUPPORTED_SHAPE;
+    if (((uintptr_t)W2 | (uintptr_t)W1 | (uintptr_t)hidden | (uintptr_t)ws) & 15) return MTV_ERR_INVALID_ARG;
     for (int d = 0; d < tree->K; ++d)
         if (tree->k_d[d] > V) return MTV_ERR_INVALID_ARG;
     const HeadsWs L = heads_ws_layout(tree, B, H, V);
@@ -333,23 +478,10 @@ extern "C" int medusa_heads_topk(const mtv_tree_t *tree, int B, int H, int V,
     auto *bb = reinterpret_cast<const __nv_bfloat16 *>(b1);
     auto *w2 = reinterpret_cast<const __nv_bfloat16 *>(W2);
     int rc;
-    if (B == 1) rc = launch_heads<1>(tree, B, H, V, h, w1, bb, w2, L, (char *)ws, st);
-    else if (B == 2) rc = launch_heads<2>(tree, B, H, V, h, w1, bb, w2, L, (char *)ws, st);
-    else rc = launch_heads<NB_MAX>(tree, B, H, V, h, w1, bb, w2, L, (char *)ws, st);
+    if (B == 1) rc = launch_heads<1>(tree, B, H, V, h, w1, bb, w2, root_tok, cand, cand_logit, tree_tok, L, (char *)ws, st);
+    else if (B == 2) rc = launch_heads<2>(tree, B, H, V, h, w1, bb, w2, root_tok, cand, cand_logit, tree_tok, L, (char *)ws, st);
+    else rc = launch_heads<NB_MAX>(tree, B, H, V, h, w1, bb, w2, root_tok, cand, cand_logit, tree_tok, L, (char *)ws, st);
     if (rc != MTV_OK) return rc;
-    const size_t smm = (size_t)tree->K * L.ctas_per_head * MTV_MAX_TOPK * 8;
-    if (smm > 200 * 1024) return MTV_ERR_UNSUPPORTED_SHAPE;
-    static bool attr_done = false;
-    if (!attr_done) {
-        MTV_CUDA_CHECK(cudaFuncSetAttribute(heads_merge_expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-        attr_done = true;
-    }
-    TapScope tap(MTV_KERNEL_HEADS_MERGE, st);
-    heads_merge_expand_kernel<<<B, tree->K * MERGE_GROUP, smm, st>>>(
-        B, tree->K, tree->T, tree->C, L.ctas_per_head,
-        reinterpret_cast<const float *>((char *)ws + L.part_val_off),
-        reinterpret_cast<const int32_t *>((char *)ws + L.part_idx_off), tree->d_kd, tree->d_cand_offset,
-        tree->d_tree_indices, root_tok, cand, cand_logit, tree_tok);
     MTV_CUDA_CHECK(cudaGetLastError());
     return MTV_OK;
 }

@@ -136,7 +136,7 @@ extern "C" int tree_build_static(int K, int n_nodes, const int32_t *node_ranks, 
     if (upload) {
         const size_t n_ti = T, n_ri = (size_t)tr->P * (K + 1), n_anc = (size_t)T * 2;
         size_t o_ti = 0, o_ri = mtv::align_up(o_ti + n_ti * 4, 16), o_anc = mtv::align_up(o_ri + n_ri * 4, 16);
-        size_t o_kd = o_anc + n_anc * 8, o_co = o_kd + MTV_MAX_K * 4, total = o_co + MTV_MAX_K * 4;
+        size_t o_kd = o_anc + n_anc * 8, o_co = o_kd + MTV_MAX_K * 4, o_err = o_co + MTV_MAX_K * 4, total = o_err + 16;
         std::vector<unsigned char> blob(total, 0);
         memcpy(blob.data() + o_ti, tr->tree_indices.data(), n_ti * 4);
         memcpy(blob.data() + o_ri, tr->retrieve.data(), n_ri * 4);
@@ -160,6 +160,7 @@ extern "C" int tree_build_static(int K, int n_nodes, const int32_t *node_ranks, 
         tr->d_anc = (const uint64_t *)(base + o_anc);
         tr->d_kd = (const int32_t *)(base + o_kd);
         tr->d_cand_offset = (const int32_t *)(base + o_co);
+        tr->d_error = (int32_t *)(base + o_err);
         tr->on_device = true;
     }
     *out = tr;
@@ -170,6 +171,13 @@ extern "C" void tree_destroy(mtv_tree_t *tree) {
     if (!tree) return;
     if (tree->d_blob) cudaFree(tree->d_blob);
     delete tree;
+}
+
+extern "C" int mtv_device_error(const mtv_tree_t *tree, int clear, int32_t *code) {
+    if (!tree || !tree->on_device || !code) return MTV_ERR_INVALID_ARG;
+    MTV_CUDA_CHECK(cudaMemcpy(code, tree->d_error, sizeof(int32_t), cudaMemcpyDeviceToHost));
+    if (clear && *code != 0) MTV_CUDA_CHECK(cudaMemset(tree->d_error, 0, sizeof(int32_t)));
+    return MTV_OK;
 }
 
 extern "C" int tree_query(const mtv_tree_t *t, mtv_tree_info *info) {
