@@ -16,15 +16,23 @@ constexpr int BN = 64;           // keys per tile
 constexpr int ATT_THREADS = 256;
 constexpr float LOG2E = 1.4426950408889634f;
 
+bool attn_tc_eligible(int D, int G);
+int launch_tree_attn_tc(const mtv_tree *tree, int B, int Hq, int Hkv, const __nv_bfloat16 *q, const __nv_bfloat16 *k,
+                        const __nv_bfloat16 *v, int64_t sb, int64_t sh, int64_t st, int Lcap, const int32_t *seq_lens,
+                        float scale_log2, float *ws_o, float *ws_ml, int nsplit, int m_rows, cudaStream_t stream);
+
 AttnWs attn_ws_layout(const mtv_tree *t, int B, int Hq, int Hkv, int D, int Lcap) {
     AttnWs w;
     const int G = Hq / Hkv;
     const int M = t->T * G;
-    const int mblocks = (M + BM - 1) / BM;
-    w.m_rows = mblocks * BM;
+    w.use_tc = attn_tc_eligible(D, G);
+    const int rows_per_cta = w.use_tc ? 256 : BM;     // query rows one CTA covers
+    const int keys_per_tile = w.use_tc ? 128 : BN;
+    const int mblocks = (M + rows_per_cta - 1) / rows_per_cta;
+    w.m_rows = mblocks * rows_per_cta;
     long ctas = (long)B * Hkv * mblocks;
     int ns = (int)(sm_count() / ctas);
-    const int tiles = (Lcap + BN - 1) / BN;
+    const int tiles = (Lcap + keys_per_tile - 1) / keys_per_tile;
     if (ns > tiles) ns = tiles;
     if (ns < 1) ns = 1;
     w.nsplit = ns;
@@ -317,15 +325,22 @@ extern "C" int tree_verify_attention(const mtv_tree_t *tree, int B, int Hq, int 
     p.B = B; p.T = tree->T; p.Hq = Hq; p.Hkv = Hkv; p.G = Hq / Hkv; p.Lcap = Lcap;
     p.nsplit = Lw.nsplit; p.m_rows = Lw.m_rows;
     cudaStream_t st = (cudaStream_t)stream;
-    const dim3 grid(Lw.nsplit, Hkv * (Lw.m_rows / BM), B);
-    const size_t smem = (size_t)4 * BN * D * 2;
-    static bool attr_done = false;
-    if (!attr_done) {
-        MTV_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_partial_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * BN * 64 * 2));
-        MTV_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_partial_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * BN * 128 * 2));
-        attr_done = true;
-    }
-    {
+    if (Lw.use_tc && scale >= 0.f) {
+        // tcgen05 path: head_dim 128, query groups of 1/2/4/8 heads
+        TapScope tap(MTV_KERNEL_ATTN_PARTIAL, st);
+        const int rc = launch_tree_attn_tc(tree, B, Hq, Hkv, p.q, p.k, p.v, stride_b, stride_h, stride_t, Lcap, seq_lens,
+                                           p.scale_log2, p.ws_o, p.ws_ml, Lw.nsplit, Lw.m_rows, st);
+        if (rc != MTV_OK) return rc;
+    } else {
+        if (Lw.use_tc) return MTV_ERR_INVALID_ARG;   // a negative scale
+        const dim3 grid(Lw.nsplit, Hkv * (Lw.m_rows / BM), B);
+        const size_t smem = (size_t)4 * BN * D * 2;
+        static bool attr_done = false;
+        if (!attr_done) {
+            MTV_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_partial_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * BN * 64 * 2));
+            MTV_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_partial_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * BN * 128 * 2));
+            attr_done = true;
+        }
         TapScope tap(MTV_KERNEL_ATTN_PARTIAL, st);
         if (D == 64) tree_attn_partial_kernel<64><<<grid, ATT_THREADS, smem, st>>>(p);
         else tree_attn_partial_kernel<128><<<grid, ATT_THREADS, smem, st>>>(p);

@@ -53,6 +53,7 @@ HeadsWs heads_ws_layout(const mtv_tree *t, int B, int H, int V);
 struct AttnWs {
     size_t o_off, ml_off, total;
     int nsplit, m_rows;
+    bool use_tc;   // head_dim 128 path on the tcgen05 tensor cores
 };
 AttnWs attn_ws_layout(const mtv_tree *t, int B, int Hq, int Hkv, int D, int Lcap);
 
