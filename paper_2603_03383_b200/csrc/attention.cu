@@ -17,22 +17,32 @@ constexpr int ATT_THREADS = 256;
 constexpr float LOG2E = 1.4426950408889634f;
 
 bool attn_tc_eligible(int D, int G);
+int attn_tc_plan(int T, int G, int B, int Hkv, int Lcap, int *n_rt_out);
 int launch_tree_attn_tc(const mtv_tree *tree, int B, int Hq, int Hkv, const __nv_bfloat16 *q, const __nv_bfloat16 *k,
                         const __nv_bfloat16 *v, int64_t sb, int64_t sh, int64_t st, int Lcap, const int32_t *seq_lens,
-                        float scale_log2, float *ws_o, float *ws_ml, int nsplit, int m_rows, cudaStream_t stream);
+                        float scale_log2, __nv_bfloat16 *out, int32_t *status, float *ws_o, float *ws_ml,
+                        cudaStream_t stream);
 
 AttnWs attn_ws_layout(const mtv_tree *t, int B, int Hq, int Hkv, int D, int Lcap) {
     AttnWs w;
     const int G = Hq / Hkv;
     const int M = t->T * G;
     w.use_tc = attn_tc_eligible(D, G);
-    const int rows_per_cta = w.use_tc ? 256 : BM;     // query rows one CTA covers
-    const int keys_per_tile = w.use_tc ? 128 : BN;
-    const int mblocks = (M + rows_per_cta - 1) / rows_per_cta;
-    w.m_rows = mblocks * rows_per_cta;
+    if (w.use_tc) {   // one launch; partials of the key splits pass through the workspace
+        int n_rt = 1;
+        w.nsplit = attn_tc_plan(t->T, G, B, Hkv, Lcap, &n_rt);
+        w.m_rows = 256;
+        const size_t slabs = w.nsplit > 1 ? (size_t)B * Hkv * n_rt * w.nsplit : 0;
+        w.o_off = 0;
+        w.ml_off = align_up(slabs * 256 * D * sizeof(float), 256);
+        w.total = align_up(w.ml_off + slabs * 256 * 2 * sizeof(float), 256) + 256;
+        return w;
+    }
+    const int mblocks = (M + BM - 1) / BM;
+    w.m_rows = mblocks * BM;
     long ctas = (long)B * Hkv * mblocks;
     int ns = (int)(sm_count() / ctas);
-    const int tiles = (Lcap + keys_per_tile - 1) / keys_per_tile;
+    const int tiles = (Lcap + BN - 1) / BN;
     if (ns > tiles) ns = tiles;
     if (ns < 1) ns = 1;
     w.nsplit = ns;
@@ -326,11 +336,13 @@ extern "C" int tree_verify_attention(const mtv_tree_t *tree, int B, int Hq, int 
     p.nsplit = Lw.nsplit; p.m_rows = Lw.m_rows;
     cudaStream_t st = (cudaStream_t)stream;
     if (Lw.use_tc && scale >= 0.f) {
-        // tcgen05 path: head_dim 128, query groups of 1/2/4/8 heads
+        // tcgen05 path: head_dim 128, query groups of 1/2/4/8 heads; one launch
         TapScope tap(MTV_KERNEL_ATTN_PARTIAL, st);
         const int rc = launch_tree_attn_tc(tree, B, Hq, Hkv, p.q, p.k, p.v, stride_b, stride_h, stride_t, Lcap, seq_lens,
-                                           p.scale_log2, p.ws_o, p.ws_ml, Lw.nsplit, Lw.m_rows, st);
+                                           p.scale_log2, p.out, status, p.ws_o, p.ws_ml, st);
         if (rc != MTV_OK) return rc;
+        MTV_CUDA_CHECK(cudaGetLastError());
+        return MTV_OK;
     } else {
         if (Lw.use_tc) return MTV_ERR_INVALID_ARG;   // a negative scale
         const dim3 grid(Lw.nsplit, Hkv * (Lw.m_rows / BM), B);

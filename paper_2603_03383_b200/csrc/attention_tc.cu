@@ -4,14 +4,23 @@
 // that shares one KV head) and a contiguous range of 128-key tiles.  Warp roles:
 //   warps 0-3 / 4-7  softmax warpgroup of row tile 0 / 1: one thread per query row reads its
 //                    row of S from tensor memory, applies the ancestor bitmask on the tiles that
-//                    overlap the tree rows, keeps a running (max, sum), writes P (bf16) back to
-//                    tensor memory over S, and finally writes the unnormalised partial
-//                    (m, l, O) of its row to the workspace;
+//                    overlap the tree rows, keeps a running (max, sum) and writes P (bf16) back
+//                    to tensor memory over S;
 //   warp 8           issues tcgen05.mma: S_t = Q_t K^T (operands in shared memory) and
 //                    O_t += P_t V (P from tensor memory, V from shared memory, N-major);
-//   warp 9           TMA producer: Q once, then K and V tiles through a ring of 32 KB slots.
+//   warp 9           TMA producer: Q once, then K and V tiles through a ring of 32 KB slots;
+//   warps 10-11      only help with the copies of the merge.
 // Tensor memory: S0 | S1 | O0 | O1, 128 fp32 columns each; P_t overlays the first 64 columns
-// of S_t.  The second kernel of attention.cu merges the partials of the key splits.
+// of S_t.  The softmax warpgroups take registers from the third warpgroup (setmaxnreg), so a
+// thread holds its whole row of S.
+//
+// The key splits of one query block are merged inside the same launch.  After its last key tile
+// a CTA parks its unnormalised partial (m, l, O) in shared memory, copies it coalesced to the
+// workspace (it stays in L2), and arrives on a counter of its query block.  When all splits of
+// the block have arrived, every CTA merges a slice of the rows from all partials, normalises
+// and writes bf16 output rows.  The launch is cooperative, so all CTAs are resident together and
+// the wait on the counter always ends; it is bounded all the same.  The counters live in the
+// tree object, start at zero and are put back to zero by the last CTA to leave.
 //
 // The running max is only raised when the new row max exceeds it by more than 8 (in log2
 // units), so O in tensor memory is rescaled rarely; P stays below 2^8.
@@ -24,7 +33,8 @@ namespace mtv {
 
 constexpr int TC_BN = 128;
 constexpr int TC_SLOTS = 5;
-constexpr int TC_THREADS = 320;
+constexpr int TC_THREADS = 384;   // 3 warpgroups: softmax 0, softmax 1, {MMA warp, TMA warp, 2 helper warps}
+constexpr int TC_SOFTMAX_THREADS = 256;
 constexpr uint32_t TC_TILE_BYTES = 128 * 128 * 2;   // one 128 x 128 bf16 tile: two 64-column halves
 constexpr uint32_t TC_HALF_BYTES = TC_TILE_BYTES / 2;
 constexpr uint32_t TC_Q_BYTES = 2 * TC_TILE_BYTES;
@@ -32,6 +42,29 @@ constexpr uint32_t TC_RING_BYTES = TC_SLOTS * TC_TILE_BYTES;
 constexpr uint32_t TC_BAR_BYTES = 256;
 constexpr uint32_t TC_SMEM_BYTES = 1024 + TC_Q_BYTES + TC_RING_BYTES + TC_BAR_BYTES;
 constexpr float TC_RESCALE_THRESHOLD = 8.f;
+constexpr int TC_MAX_SPLITS = 32;
+constexpr int TC_MAX_GROUPS = 256;   // merge counters available in the tree object
+
+// Register rebalancing.  The CTA's pool is what the launch allocates: TC_THREADS threads at the
+// per-thread count the compiler derives from the launch bounds (65536 / 384 rounded down to a
+// multiple of 8 = 168).  setmaxnreg.inc blocks until the pool has the registers, so the three
+// warpgroups' targets must not add up to more than the pool: 2 x 216 + 72 = 3 x 168.
+constexpr int TC_REGS_LAUNCH = 168, TC_REGS_SOFTMAX = 216, TC_REGS_OTHER = 72;
+static_assert(2 * TC_REGS_SOFTMAX + TC_REGS_OTHER <= 3 * TC_REGS_LAUNCH, "setmaxnreg targets exceed the CTA's register pool");
+static_assert(TC_REGS_LAUNCH * TC_THREADS <= 65536, "launch register count does not fit the register file");
+
+// After the last key tile the Q / K / V buffers are reused:
+//   [0, PARK_O)            parked O, 256 rows of TC_O_STRIDE floats (528 bytes: conflict-free 16-byte stores)
+//   [PARK_O, +2048)        parked (m, l) per row
+//   [.., +WBUF)            (m, l) of every split for the rows this CTA merges, then their weights
+//   [.., +1024)            1 / l of the merged rows
+constexpr int TC_O_STRIDE = 132;
+constexpr uint32_t TC_PARK_O_BYTES = 256 * TC_O_STRIDE * 4;
+constexpr uint32_t TC_PARK_ML_OFF = TC_PARK_O_BYTES;
+constexpr uint32_t TC_WBUF_OFF = TC_PARK_ML_OFF + 256 * 8;
+constexpr uint32_t TC_WBUF_ENTRIES = 256 + TC_MAX_SPLITS;
+constexpr uint32_t TC_ROWINV_OFF = TC_WBUF_OFF + TC_WBUF_ENTRIES * 8;
+static_assert(TC_ROWINV_OFF + 256 * 4 <= TC_Q_BYTES + TC_RING_BYTES, "merge buffers must fit the tile buffers");
 
 // barrier slots (8 bytes each) inside the barrier region
 enum { BAR_Q = 0, BAR_KV_FULL = 1, BAR_KV_EMPTY = BAR_KV_FULL + TC_SLOTS, BAR_S = BAR_KV_EMPTY + TC_SLOTS,
@@ -46,10 +79,14 @@ constexpr uint32_t IDESC_PV = IDESC_BASE | (1u << 16);  // B (= V) N-major
 struct TcParams {
     const int32_t *seq_lens;
     const uint64_t *anc;   // [T][2]
-    float *ws_o, *ws_ml;
+    __nv_bfloat16 *out;    // [B][T][Hq][128]
+    float *ws_o;           // [groups][nsplit][256][128] partial O (only when nsplit > 1)
+    float2 *ws_ml;         // [groups][nsplit][256] partial (m, l)
+    int32_t *arrive, *depart;   // [groups] merge counters, zero between calls
+    int32_t *status;       // [B] or null
     int32_t *dev_error;
     float scale_log2;
-    int T, G, Hkv, Lcap, nsplit, m_rows, n_rt, M_rows;
+    int T, G, Hq, Hkv, Lcap, nsplit, n_rt, M_rows;
 };
 
 // 128-byte-swizzled shared-memory operand descriptor.
@@ -66,6 +103,14 @@ __device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr) { return smem_de
 // N-major operand: 64-column halves TC_HALF_BYTES apart, 8-key groups 1024 bytes apart
 __device__ __forceinline__ uint64_t desc_nmajor(uint32_t saddr) { return smem_desc(saddr, TC_HALF_BYTES, 1024); }
 
+// Register rebalancing between warpgroups (all four warps of a warpgroup execute it).
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+
+// CTA-wide barrier usable from the diverged warp roles (every thread of the CTA arrives on it,
+// from whichever copy of the epilogue it runs).
+__device__ __forceinline__ void cta_sync() { asm volatile("bar.sync 1, %0;" ::"n"(TC_THREADS) : "memory"); }
+
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -76,6 +121,192 @@ __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
+__device__ __forceinline__ int ld_acquire(const int32_t *p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Developer timeline (compiled out unless MTV_TRACE is defined): lane 0 of the calling warp
+// stores the SM cycle counter of event `id` for this CTA.
+#ifdef MTV_TRACE
+__device__ long long *g_trace = nullptr;   // [ctas][64]
+#define TRACE_CTA ((size_t)(blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x)
+#define TRACE(id)                                                                      \
+    do {                                                                               \
+        if (g_trace && (threadIdx.x % 32) == 0) g_trace[TRACE_CTA * 64 + (id)] = clock64(); \
+    } while (0)
+#else
+#define TRACE(id)
+#endif
+
+// What the epilogue needs from the main body.
+struct TcCtx {
+    unsigned char *tiles;   // 1024-byte aligned base of the tile buffers (generic address)
+    uint32_t bars;          // shared address of the barrier region
+    volatile int *abort_flag;
+    uint32_t tmem;
+    int nt, split, rows0, g, b, cnt;
+    bool final_committed;
+};
+
+// Everything after the last key tile; instantiated once for the softmax warpgroups (which have
+// the registers to keep many loads in flight) and once for the third warpgroup.
+template <bool SOFTMAX>
+__device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    float *park_o = reinterpret_cast<float *>(c.tiles);
+    float2 *park_ml = reinterpret_cast<float2 *>(c.tiles + TC_PARK_ML_OFF);
+    float2 *wbuf = reinterpret_cast<float2 *>(c.tiles + TC_WBUF_OFF);
+    float *rowinv = reinterpret_cast<float *>(c.tiles + TC_ROWINV_OFF);
+    auto bar = [&](int i) { return c.bars + (uint32_t)i * 8u; };
+
+    ptx::tc_fence_before();
+    cta_sync();   // every role is done; partials are parked
+    if (*c.abort_flag) {
+        // A bounded wait ran out: raise the sticky error, give outstanding copies and tensor-core
+        // work one more bounded chance to finish.  The CTA still takes part in the merge so that
+        // the other splits never wait for it; the error word tells the host the output is invalid.
+        if (threadIdx.x == 0) atomicExch(p.dev_error, MTV_ERR_TIMEOUT);
+        if (!SOFTMAX) {
+            if (warp == 9 && lane == 0) {
+                ptx::mbar_wait(bar(BAR_Q), 0);
+                for (int s = 0; s < TC_SLOTS; ++s) { ptx::mbar_wait(bar(BAR_KV_FULL + s), 0); ptx::mbar_wait(bar(BAR_KV_FULL + s), 1); }
+            }
+            if (warp == 8) {
+                if (!c.final_committed && lane == 0) ptx::tc_commit(bar(BAR_FINAL));
+                __syncwarp();
+                ptx::mbar_wait(bar(BAR_FINAL), 0);
+            }
+        }
+        cta_sync();
+    }
+    if (warp == 0) TRACE(44);   // partial parked
+
+    const int act_rows = c.nt * 128;
+    const int nsplit = p.nsplit;
+    const int grp = blockIdx.z * gridDim.y + blockIdx.y;
+    if (nsplit == 1) {
+        // the partial is the result: normalise and store
+        for (int item = threadIdx.x; item < act_rows * 32; item += TC_THREADS) {
+            const int row = item / 32, c4 = item % 32, r = c.rows0 + row;
+            if (r >= p.M_rows) continue;
+            const float4 v = *reinterpret_cast<const float4 *>(park_o + row * TC_O_STRIDE + c4 * 4);
+            const float inv = 1.f / park_ml[row].y;
+            uint2 packed;
+            packed.x = pack2_bf16(v.x * inv, v.y * inv);
+            packed.y = pack2_bf16(v.z * inv, v.w * inv);
+            const int node = r / p.G, hq = c.g * p.G + r % p.G;
+            *reinterpret_cast<uint2 *>(p.out + (((size_t)c.b * p.T + node) * p.Hq + hq) * 128 + c4 * 4) = packed;
+        }
+    } else {
+        // ---- publish the partial
+        const size_t slab = ((size_t)grp * nsplit + c.split) * 256;
+        for (int idx = threadIdx.x; idx < act_rows * 32; idx += TC_THREADS) {
+            const int row = idx / 32, c4 = idx % 32;
+            *reinterpret_cast<float4 *>(p.ws_o + (slab + row) * 128 + c4 * 4) =
+                *reinterpret_cast<const float4 *>(park_o + row * TC_O_STRIDE + c4 * 4);
+        }
+        for (int row = threadIdx.x; row < act_rows; row += TC_THREADS) p.ws_ml[slab + row] = park_ml[row];
+        cta_sync();
+        if (threadIdx.x == 0) {
+            __threadfence();   // cumulative: covers the CTA's stores ordered before the barrier
+            atomicAdd(p.arrive + grp, 1);
+            const long long t0 = clock64();
+            while (ld_acquire(p.arrive + grp) < nsplit)
+                if (clock64() - t0 > ptx::WAIT_CYCLE_LIMIT) { atomicExch(p.dev_error, MTV_ERR_TIMEOUT); break; }
+        }
+        cta_sync();
+        if (warp == 0) TRACE(45);   // all splits arrived
+
+        // ---- merge rows [row_begin, row_begin + n_my) of the query block from all splits
+        const int rows_per = (act_rows + nsplit - 1) / nsplit;
+        const int row_begin = c.split * rows_per;
+        const int n_my = max(0, min(act_rows, row_begin + rows_per) - row_begin);
+        const size_t src0 = (size_t)grp * nsplit * 256 + row_begin;   // + s * 256 + local row
+        for (int idx = threadIdx.x; idx < n_my * nsplit; idx += TC_THREADS) {
+            const int rl = idx / nsplit, s = idx - rl * nsplit;
+            wbuf[idx] = __ldcg(p.ws_ml + src0 + (size_t)s * 256 + rl);
+        }
+        // Thread tid of the softmax warpgroups owns the items (row, 4 columns) tid, tid + 256, ...;
+        // its loads of all splits are independent of the weights, so they go out first.
+        constexpr int NBUF = 36;
+        float4 v[NBUF];
+        const int n_items = n_my * 32;
+        const int my_items = SOFTMAX && (int)threadIdx.x < n_items ? (n_items - (int)threadIdx.x + TC_SOFTMAX_THREADS - 1) / TC_SOFTMAX_THREADS : 0;
+        const int n_pairs = my_items * nsplit;     // pair q = k * nsplit + s: item k of this thread, split s
+        auto pair_src = [&](int q) {
+            const int k = q / nsplit, s = q - k * nsplit;
+            const int item = threadIdx.x + k * TC_SOFTMAX_THREADS;
+            return reinterpret_cast<const float4 *>(p.ws_o + (src0 + (size_t)s * 256 + item / 32) * 128 + (item % 32) * 4);
+        };
+        if (SOFTMAX) {
+#pragma unroll
+            for (int u = 0; u < NBUF; ++u)
+                if (u < n_pairs) v[u] = __ldcg(pair_src(u));
+        }
+        cta_sync();
+        for (int rl = threadIdx.x; rl < n_my; rl += TC_THREADS) {
+            float m = -INFINITY;
+            for (int s = 0; s < nsplit; ++s) m = fmaxf(m, wbuf[rl * nsplit + s].x);
+            float lsum = 0.f;
+            for (int s = 0; s < nsplit; ++s) {
+                const float2 ml = wbuf[rl * nsplit + s];
+                const float w = ml.x == -INFINITY ? 0.f : ex2(ml.x - m);
+                lsum += w * ml.y;
+                wbuf[rl * nsplit + s].x = w;
+            }
+            rowinv[rl] = 1.f / lsum;
+        }
+        cta_sync();
+        if (SOFTMAX) {
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int q0 = 0; q0 < n_pairs; q0 += NBUF) {
+                if (q0 > 0) {
+#pragma unroll
+                    for (int u = 0; u < NBUF; ++u)
+                        if (q0 + u < n_pairs) v[u] = __ldcg(pair_src(q0 + u));
+                }
+#pragma unroll
+                for (int u = 0; u < NBUF; ++u) {
+                    const int q = q0 + u;
+                    if (q < n_pairs) {
+                        const int k = q / nsplit, s = q - k * nsplit;
+                        const int item = threadIdx.x + k * TC_SOFTMAX_THREADS;
+                        const int rl = item / 32, c4 = item % 32;
+                        const float w = wbuf[rl * nsplit + s].x;
+                        acc.x = fmaf(w, v[u].x, acc.x); acc.y = fmaf(w, v[u].y, acc.y);
+                        acc.z = fmaf(w, v[u].z, acc.z); acc.w = fmaf(w, v[u].w, acc.w);
+                        if (s == nsplit - 1) {
+                            const int r = c.rows0 + row_begin + rl;
+                            if (r < p.M_rows) {
+                                const float inv = rowinv[rl];
+                                uint2 packed;
+                                packed.x = pack2_bf16(acc.x * inv, acc.y * inv);
+                                packed.y = pack2_bf16(acc.z * inv, acc.w * inv);
+                                const int node = r / p.G, hq = c.g * p.G + r % p.G;
+                                *reinterpret_cast<uint2 *>(p.out + (((size_t)c.b * p.T + node) * p.Hq + hq) * 128 + c4 * 4) = packed;
+                            }
+                            acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+                    }
+                }
+            }
+        }
+        if (warp == 0) TRACE(46);   // merge done
+        // the last CTA of the query block to get here puts the counters back to zero
+        if (threadIdx.x == 0 && atomicAdd(p.depart + grp, 1) == nsplit - 1) {
+            p.arrive[grp] = 0;
+            p.depart[grp] = 0;
+            __threadfence();
+        }
+    }
+    if (!SOFTMAX && warp == 8) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(c.tmem, 512);
+    }
+    if (warp == 0) TRACE(47);
+}
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
@@ -85,7 +316,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     const int g = blockIdx.y / p.n_rt, rt = blockIdx.y % p.n_rt;
     const int b = blockIdx.z;
     const int L = p.seq_lens[b];
-    if (L + p.T > p.Lcap) return;   // reported by the combine kernel
+    const bool reporter = blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0;
+    if (L + p.T > p.Lcap) {         // the same for every CTA of the query block: nobody waits for anybody
+        if (reporter && p.status) p.status[b] = MTV_ERR_CAPACITY;
+        return;
+    }
+    if (reporter && p.status) p.status[b] = MTV_OK;
     const int n_keys = L + p.T;
     const int tiles = (n_keys + TC_BN - 1) / TC_BN;
     const int base_cnt = tiles / p.nsplit, rem = tiles % p.nsplit;
@@ -93,14 +329,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     const int cnt = base_cnt + (split < rem ? 1 : 0);
     const int rows0 = rt * 256;
     const int nt = p.M_rows - rows0 > 128 ? 2 : 1;
-    const size_t slab = (((size_t)b * p.Hkv + g) * p.nsplit + split) * p.m_rows + rows0;
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-
-    if (cnt == 0) {   // no keys for this split: an empty partial
-        for (int r = threadIdx.x; r < nt * 128; r += TC_THREADS)
-            *reinterpret_cast<float2 *>(p.ws_ml + (slab + r) * 2) = make_float2(-INFINITY, 0.f);
-        return;
-    }
+    if (warp == 0) TRACE(0);
 
     // carve shared memory (tiles need 1024-byte alignment for the 128-byte swizzle)
     const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -108,12 +338,27 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     const uint32_t q_smem = raw + pad;
     const uint32_t ring = q_smem + TC_Q_BYTES;
     const uint32_t bars = ring + TC_RING_BYTES;
-    unsigned char *bar_region = smem_raw + pad + TC_Q_BYTES + TC_RING_BYTES;
+    unsigned char *tiles_gen = smem_raw + pad;
+    unsigned char *bar_region = tiles_gen + TC_Q_BYTES + TC_RING_BYTES;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(bar_region + BAR_COUNT * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bar_region + BAR_COUNT * 8 + 4);
     auto bar = [&](int i) { return bars + (uint32_t)i * 8u; };
+    float *park_o = reinterpret_cast<float *>(tiles_gen);
+    float2 *park_ml = reinterpret_cast<float2 *>(tiles_gen + TC_PARK_ML_OFF);
 
-    if (threadIdx.x == 0) {
+    // One K or V tile into ring slot (i mod TC_SLOTS): i = 2j is K of key tile j, i = 2j + 1 is V.
+    auto issue_kv = [&](int i) {
+        const int slot = i % TC_SLOTS;
+        const CUtensorMap *map = (i & 1) ? &v_map : &k_map;
+        ptx::mbar_arrive_expect_tx(bar(BAR_KV_FULL + slot), TC_TILE_BYTES);
+        for (int half = 0; half < 2; ++half)
+            ptx::tma_load_4d(ring + slot * TC_TILE_BYTES + half * TC_HALF_BYTES, map, bar(BAR_KV_FULL + slot), half * 64,
+                             (t_begin + i / 2) * TC_BN, g, b);
+    };
+    const int n_loads = 2 * cnt;
+    const int n_early = min(n_loads, TC_SLOTS);   // loads that need no free slot: issued before the CTA syncs
+
+    if (warp == 9 && lane == 0) {
         ptx::mbar_init(bar(BAR_Q), 1);
         for (int s = 0; s < TC_SLOTS; ++s) { ptx::mbar_init(bar(BAR_KV_FULL + s), 1); ptx::mbar_init(bar(BAR_KV_EMPTY + s), 1); }
         for (int t = 0; t < 2; ++t) {
@@ -124,221 +369,255 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
         ptx::mbar_init(bar(BAR_FINAL), 1);
         ptx::fence_mbar_init();
         *abort_flag = 0;
-    }
-    if (warp == 8) {
-        ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t *>(tmem_slot)), 512);
-        ptx::tmem_relinquish();
-    }
-    if (warp == 9 && lane == 0) {
-        ptx::prefetch_tensormap(&q_map);
-        ptx::prefetch_tensormap(&k_map);
-        ptx::prefetch_tensormap(&v_map);
-    }
-    ptx::tc_fence_before();
-    __syncthreads();
-    ptx::tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
-
-    if (warp == 9) {
-        // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        if (cnt > 0) {
+            // first K tile, then Q, then the rest: the first MMA needs K_0 and Q
+            issue_kv(0);
             ptx::mbar_arrive_expect_tx(bar(BAR_Q), nt * TC_TILE_BYTES);
             for (int t = 0; t < nt; ++t)
                 for (int half = 0; half < 2; ++half)
                     ptx::tma_load_4d(q_smem + t * TC_TILE_BYTES + half * TC_HALF_BYTES, &q_map, bar(BAR_Q), half * 64,
                                      g * p.G, (rows0 + t * 128) / p.G, b);
+            for (int i = 1; i < n_early; ++i) issue_kv(i);
         }
-        for (int i = 0; i < 2 * cnt && !*abort_flag; ++i) {
-            const int slot = i % TC_SLOTS, use = i / TC_SLOTS, j = i / 2;
-            if (use > 0 && !ptx::mbar_wait(bar(BAR_KV_EMPTY + slot), (use - 1) & 1)) { *abort_flag = 1; break; }
-            if (lane == 0) {
-                const CUtensorMap *map = (i & 1) ? &v_map : &k_map;
-                ptx::mbar_arrive_expect_tx(bar(BAR_KV_FULL + slot), TC_TILE_BYTES);
-                for (int half = 0; half < 2; ++half)
-                    ptx::tma_load_4d(ring + slot * TC_TILE_BYTES + half * TC_HALF_BYTES, map, bar(BAR_KV_FULL + slot),
-                                     half * 64, (t_begin + j) * TC_BN, g, b);
-            }
-            __syncwarp();
-        }
-    } else if (warp == 8) {
-        // ------------------------------------------------------------ MMA issuer
-        auto issue_S = [&](int t, int j) {
-            const uint32_t kbase = ring + ((2 * j) % TC_SLOTS) * TC_TILE_BYTES;
-            const uint32_t qbase = q_smem + t * TC_TILE_BYTES;
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-                const uint32_t off = (kk / 4) * TC_HALF_BYTES + (kk % 4) * 32;
-                ptx::mma_ss(tmem + t * 128, desc_kmajor(qbase + off), desc_kmajor(kbase + off), IDESC_QK, kk > 0);
-            }
-        };
-        auto issue_PV = [&](int t, int j) {
-            const uint32_t vbase = ring + ((2 * j + 1) % TC_SLOTS) * TC_TILE_BYTES;
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-                ptx::mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, desc_nmajor(vbase + kk * 2048), IDESC_PV,
-                            j > 0 || kk > 0);
-        };
-        auto wait_kv = [&](int i) { return ptx::mbar_wait(bar(BAR_KV_FULL + i % TC_SLOTS), (i / TC_SLOTS) & 1); };
-        bool ok = ptx::mbar_wait(bar(BAR_Q), 0) && wait_kv(0);
-        if (ok) {
-            ptx::tc_fence_after();
-            if (lane == 0) {
-                issue_S(0, 0);
-                ptx::tc_commit(bar(BAR_S + 0));
-                if (nt == 2) { issue_S(1, 0); ptx::tc_commit(bar(BAR_S + 1)); }
-                ptx::tc_commit(bar(BAR_KV_EMPTY + 0));
-            }
-            __syncwarp();
-        }
-        for (int j = 0; ok && j < cnt && !*abort_flag; ++j) {
-            const bool more = j + 1 < cnt;
-            ok = wait_kv(2 * j + 1) && ptx::mbar_wait(bar(BAR_P + 0), j & 1);
-            if (!ok) break;
-            ptx::tc_fence_after();
-            if (lane == 0) { issue_PV(0, j); ptx::tc_commit(bar(BAR_O + 0)); }
-            __syncwarp();
-            if (more) {
-                ok = wait_kv(2 * j + 2);
-                if (!ok) break;
-                ptx::tc_fence_after();
-                if (lane == 0) { issue_S(0, j + 1); ptx::tc_commit(bar(BAR_S + 0)); }
+    }
+    if (warp == 8) {
+        ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t *>(tmem_slot)), 512);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    if (warp == 0) TRACE(1);
+
+    TcCtx ctx;
+    ctx.tiles = tiles_gen; ctx.bars = bars; ctx.abort_flag = abort_flag; ctx.tmem = *tmem_slot;
+    ctx.nt = nt; ctx.split = split; ctx.rows0 = rows0; ctx.g = g; ctx.b = b; ctx.cnt = cnt;
+    ctx.final_committed = false;
+    const uint32_t tmem = ctx.tmem;
+
+    if (warp >= 8) {
+        reg_dec<TC_REGS_OTHER>();   // the whole third warpgroup gives registers to the softmax warpgroups
+        if (warp == 9) {
+            // ------------------------------------------------------------ TMA producer (the rest of the tiles)
+            for (int i = n_early; i < n_loads && !*abort_flag; ++i) {
+                const int slot = i % TC_SLOTS, use = i / TC_SLOTS;
+                if (!ptx::mbar_wait(bar(BAR_KV_EMPTY + slot), (use - 1) & 1)) { *abort_flag = 1; break; }
+                if (lane == 0) issue_kv(i);
                 __syncwarp();
             }
-            if (nt == 2) {
-                ok = ptx::mbar_wait(bar(BAR_P + 1), j & 1);
-                if (!ok) break;
-                ptx::tc_fence_after();
-                if (lane == 0) { issue_PV(1, j); ptx::tc_commit(bar(BAR_O + 1)); }
-                __syncwarp();
-            }
-            if (lane == 0) {
-                ptx::tc_commit(bar(BAR_KV_EMPTY + (2 * j + 1) % TC_SLOTS));   // V_j is free once its MMAs are done
-                if (more) {
-                    if (nt == 2) { issue_S(1, j + 1); ptx::tc_commit(bar(BAR_S + 1)); }
-                    ptx::tc_commit(bar(BAR_KV_EMPTY + (2 * j + 2) % TC_SLOTS));
+        } else if (warp == 8) {
+            // ------------------------------------------------------------ MMA issuer
+            auto issue_S = [&](int t, int j) {
+                const uint32_t kbase = ring + ((2 * j) % TC_SLOTS) * TC_TILE_BYTES;
+                const uint32_t qbase = q_smem + t * TC_TILE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t off = (kk / 4) * TC_HALF_BYTES + (kk % 4) * 32;
+                    ptx::mma_ss(tmem + t * 128, desc_kmajor(qbase + off), desc_kmajor(kbase + off), IDESC_QK, kk > 0);
                 }
-            }
-            __syncwarp();
-        }
-        if (!ok) *abort_flag = 1;
-    } else if (warp / 4 < nt) {
-        // ------------------------------------------------------------ softmax warpgroup of row tile t
-        const int t = warp / 4;
-        const int row = (warp % 4) * 32 + lane;
-        const int r = rows0 + t * 128 + row;
-        uint64_t alo = 0, ahi = 0;
-        if (r < p.M_rows) { alo = p.anc[(r / p.G) * 2]; ahi = p.anc[(r / p.G) * 2 + 1]; }
-        const uint32_t t_s = tmem + ((uint32_t)((warp % 4) * 32) << 16) + t * 128;
-        const uint32_t t_o = tmem + ((uint32_t)((warp % 4) * 32) << 16) + 256 + t * 128;
-        float m_used = -INFINITY, l = 0.f;
-        bool ok = true;
-        for (int j = 0; j < cnt && !*abort_flag; ++j) {
-            ok = ptx::mbar_wait(bar(BAR_S + t), j & 1);
-            if (!ok) break;
-            ptx::tc_fence_after();
-            uint32_t s[4][32];
+            };
+            auto issue_PV = [&](int t, int j) {
+                const uint32_t vbase = ring + ((2 * j + 1) % TC_SLOTS) * TC_TILE_BYTES;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) ptx::tmem_ld32(t_s + c * 32, s[c]);
-            ptx::tmem_ld_wait();
-            const int key0 = (t_begin + j) * TC_BN;
-            if (key0 + TC_BN > L) {
-                // tile overlaps the tree rows (or the end of the cache): column c is key key0 + c
-                const int off = L - key0;   // first tree row's column (may be negative)
+                for (int kk = 0; kk < 8; ++kk)
+                    ptx::mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, desc_nmajor(vbase + kk * 2048), IDESC_PV,
+                                j > 0 || kk > 0);
+            };
+            auto wait_kv = [&](int i) { return ptx::mbar_wait(bar(BAR_KV_FULL + i % TC_SLOTS), (i / TC_SLOTS) & 1); };
+            bool ok = cnt == 0 || (wait_kv(0) && ptx::mbar_wait(bar(BAR_Q), 0));
+            if (ok && cnt > 0) {
+                TRACE(2);   // Q and K_0 landed
+                ptx::tc_fence_after();
+                if (lane == 0) {
+                    issue_S(0, 0);
+                    ptx::tc_commit(bar(BAR_S + 0));
+                    if (nt == 2) { issue_S(1, 0); ptx::tc_commit(bar(BAR_S + 1)); }
+                    ptx::tc_commit(bar(BAR_KV_EMPTY + 0));
+                }
+                __syncwarp();
+            }
+            for (int j = 0; ok && j < cnt && !*abort_flag; ++j) {
+                const bool more = j + 1 < cnt;
+                ok = wait_kv(2 * j + 1);
+                if (!ok) break;
+                {
+                    // Rows of the V tile past the last valid key hold whatever the cache holds there; their
+                    // P is zero, but 0 * NaN would still poison O: clear them before the tensor core reads.
+                    const int valid = n_keys - (t_begin + j) * TC_BN;
+                    if (valid < TC_BN) {
+                        unsigned char *vt = tiles_gen + TC_Q_BYTES + ((2 * j + 1) % TC_SLOTS) * TC_TILE_BYTES;
+                        for (int e = lane; e < (TC_BN - valid) * 16; e += 32) {
+                            const int row = valid + e / 16, c16 = e % 16;     // 16 x 16 bytes per row: 8 per half
+                            *reinterpret_cast<uint4 *>(vt + (c16 / 8) * TC_HALF_BYTES + row * 128 + (c16 % 8) * 16) =
+                                make_uint4(0u, 0u, 0u, 0u);
+                        }
+                        ptx::fence_proxy_async();
+                        __syncwarp();
+                    }
+                }
+                ok = ptx::mbar_wait(bar(BAR_P + 0), j & 1);
+                if (!ok) break;
+                ptx::tc_fence_after();
+                if (lane == 0) { issue_PV(0, j); ptx::tc_commit(bar(BAR_O + 0)); }
+                __syncwarp();
+                if (more) {
+                    ok = wait_kv(2 * j + 2);
+                    if (!ok) break;
+                    ptx::tc_fence_after();
+                    if (lane == 0) { issue_S(0, j + 1); ptx::tc_commit(bar(BAR_S + 0)); }
+                    __syncwarp();
+                }
+                if (nt == 2) {
+                    ok = ptx::mbar_wait(bar(BAR_P + 1), j & 1);
+                    if (!ok) break;
+                    ptx::tc_fence_after();
+                    if (lane == 0) { issue_PV(1, j); ptx::tc_commit(bar(BAR_O + 1)); }
+                    __syncwarp();
+                }
+                if (lane == 0) {
+                    ptx::tc_commit(bar(BAR_KV_EMPTY + (2 * j + 1) % TC_SLOTS));   // V_j is free once its MMAs are done
+                    if (more) {
+                        if (nt == 2) { issue_S(1, j + 1); ptx::tc_commit(bar(BAR_S + 1)); }
+                        ptx::tc_commit(bar(BAR_KV_EMPTY + (2 * j + 2) % TC_SLOTS));
+                    }
+                }
+                __syncwarp();
+            }
+            if (ok && cnt > 0 && !*abort_flag) {
+                if (lane == 0) ptx::tc_commit(bar(BAR_FINAL));   // follows every tensor-core operation issued
+                __syncwarp();
+                ctx.final_committed = true;
+            }
+            if (!ok) *abort_flag = 1;
+        }
+        tc_epilogue<false>(p, ctx);
+    } else {
+        reg_inc<TC_REGS_SOFTMAX>();
+        if (warp / 4 < nt) {
+            // ------------------------------------------------------------ softmax warpgroup of row tile t
+            const int t = warp / 4;
+            const int row = (warp % 4) * 32 + lane;
+            const int r = rows0 + t * 128 + row;
+            uint64_t alo = 0, ahi = 0;
+            if (r < p.M_rows) { alo = p.anc[(r / p.G) * 2]; ahi = p.anc[(r / p.G) * 2 + 1]; }
+            const uint32_t t_s = tmem + ((uint32_t)((warp % 4) * 32) << 16) + t * 128;
+            const uint32_t t_o = tmem + ((uint32_t)((warp % 4) * 32) << 16) + 256 + t * 128;
+            float m_used = -INFINITY, l = 0.f;
+            bool ok = true;
+            // visibility of the tree rows as 32-bit words: word q covers tree rows 32q .. 32q+31
+            auto anc_word = [&](int q) -> uint32_t {
+                if (q < 0) return 0xffffffffu;     // prefix rows are visible to every node
+                if (q == 0) return (uint32_t)alo;
+                if (q == 1) return (uint32_t)(alo >> 32);
+                if (q == 2) return (uint32_t)ahi;
+                if (q == 3) return (uint32_t)(ahi >> 32);
+                return 0u;                         // past the tree rows: nothing
+            };
+            for (int j = 0; j < cnt && !*abort_flag; ++j) {
+                ok = ptx::mbar_wait(bar(BAR_S + t), j & 1);
+                if (!ok) break;
+                if (warp % 4 == 0 && j < 6) TRACE(8 + t * 16 + j * 2);       // S_t(j) ready
+                ptx::tc_fence_after();
+                // ---- the whole row of S in registers (raw scores; the scale is positive)
+                uint32_t sr[4][32];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) ptx::tmem_ld32(t_s + c * 32, sr[c]);
+                ptx::tmem_ld_wait();
+                const int key0 = (t_begin + j) * TC_BN;
+                if (key0 + TC_BN > L) {
+                    // tile overlaps the tree rows or the end of the cache: bit e of vis is column 32c + e
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const int a0 = key0 + c * 32 - L;        // tree row of the chunk's first column
+                        const int q = a0 >> 5, sh = a0 & 31;     // floor division
+                        const uint32_t vis = __funnelshift_r(anc_word(q), anc_word(q + 1), sh);
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (!((vis >> e) & 1u)) sr[c][e] = 0xff800000u;   // -inf
+                    }
+                }
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        const int a = c * 32 + e - off;
-                        bool vis;
-                        if (a < 0) vis = true;
-                        else if (a < 64) vis = (alo >> a) & 1ull;
-                        else if (a < 128) vis = (ahi >> (a - 64)) & 1ull;
-                        else vis = false;
-                        if (!vis) s[c][e] = 0xff800000u;   // -inf
+                    for (int e = 0; e < 32; e += 4) {
+                        mx0 = fmaxf(mx0, __uint_as_float(sr[c][e]));
+                        mx1 = fmaxf(mx1, __uint_as_float(sr[c][e + 1]));
+                        mx2 = fmaxf(mx2, __uint_as_float(sr[c][e + 2]));
+                        mx3 = fmaxf(mx3, __uint_as_float(sr[c][e + 3]));
                     }
-            }
-            float mx = -INFINITY;
+                const float mxs = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
+                const float m_new = (j == 0 || mxs > m_used + TC_RESCALE_THRESHOLD) ? mxs : m_used;
+                // O holds sums relative to m_used: rescale it when the reference moves (rare)
+                const bool need = j > 0 && m_new != m_used && m_used != -INFINITY;
+                if (__any_sync(0xffffffffu, need)) {
+                    ok = ptx::mbar_wait(bar(BAR_O + t), (j - 1) & 1);
+                    if (!ok) break;
+                    ptx::tc_fence_after();
+                    const float alpha = need ? ex2(m_used - m_new) : 1.f;
+#pragma unroll 1
+                    for (int c = 0; c < 8; ++c) {
+                        uint32_t o[16];
+                        ptx::tmem_ld16(t_o + c * 16, o);
+                        ptx::tmem_ld_wait();
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-#pragma unroll
-                for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(s[c][e]));
-            const float mxs = mx * p.scale_log2;
-            const float m_new = (j == 0 || mxs > m_used + TC_RESCALE_THRESHOLD) ? mxs : m_used;
-            // O holds sums relative to m_used: rescale it when the reference moves (rare)
-            const bool need = j > 0 && m_new != m_used && m_used != -INFINITY;
-            if (__any_sync(0xffffffffu, need)) {
-                ok = ptx::mbar_wait(bar(BAR_O + t), (j - 1) & 1);
-                if (!ok) break;
-                ptx::tc_fence_after();
-                const float alpha = need ? ex2(m_used - m_new) : 1.f;
+                        for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                        ptx::tmem_st16(t_o + c * 16, o);
+                    }
+                    ptx::tmem_st_wait();
+                    l *= alpha;
+                }
+                m_used = m_new;
+                const float m_eff = m_used == -INFINITY ? 0.f : m_used;
+                // ---- P = exp2(scale * S - m), row sum, bf16 P over the first 64 columns of S
+                float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    uint32_t o[32];
-                    ptx::tmem_ld32(t_o + c * 32, o);
-                    ptx::tmem_ld_wait();
+                    uint32_t pk[16];
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                    ptx::tmem_st32(t_o + c * 32, o);
+                    for (int e = 0; e < 16; e += 2) {
+                        const float p0 = ex2(fmaf(__uint_as_float(sr[c][2 * e]), p.scale_log2, -m_eff));
+                        const float p1 = ex2(fmaf(__uint_as_float(sr[c][2 * e + 1]), p.scale_log2, -m_eff));
+                        const float p2 = ex2(fmaf(__uint_as_float(sr[c][2 * e + 2]), p.scale_log2, -m_eff));
+                        const float p3 = ex2(fmaf(__uint_as_float(sr[c][2 * e + 3]), p.scale_log2, -m_eff));
+                        l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+                        pk[e] = pack2_bf16(p0, p1);
+                        pk[e + 1] = pack2_bf16(p2, p3);
+                    }
+                    ptx::tmem_st16(t_s + c * 16, pk);
                 }
+                l += (l0 + l1) + (l2 + l3);
                 ptx::tmem_st_wait();
-                l *= alpha;
+                ptx::tc_fence_before();
+                ptx::mbar_arrive(bar(BAR_P + t));
+                if (warp % 4 == 0 && j < 6) TRACE(9 + t * 16 + j * 2);       // P_t(j) written
             }
-            m_used = m_new;
-            const float m_eff = m_used == -INFINITY ? 0.f : m_used;
+            // ---- park the partial of this row in shared memory
+            float *dst = park_o + (t * 128 + row) * TC_O_STRIDE;
+            if (cnt > 0) {
+                // every tensor-core read of the tile buffers must be over before they are reused
+                if (ok && !*abort_flag) ok = ptx::mbar_wait(bar(BAR_FINAL), 0);
+                if (warp % 4 == 0) TRACE(40 + t);                            // all tensor-core work done
+                if (ok && !*abort_flag) {
+                    ptx::tc_fence_after();
+#pragma unroll 1
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t o[32];
+                        ptx::tmem_ld32(t_o + c * 32, o);
+                        ptx::tmem_ld_wait();
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const float p0 = ex2(fmaf(__uint_as_float(s[c][2 * e]), p.scale_log2, -m_eff));
-                    const float p1 = ex2(fmaf(__uint_as_float(s[c][2 * e + 1]), p.scale_log2, -m_eff));
-                    l += p0 + p1;
-                    pk[e] = pack2_bf16(p0, p1);
+                        for (int e = 0; e < 32; e += 4)
+                            *reinterpret_cast<uint4 *>(dst + c * 32 + e) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
+                    }
                 }
-                ptx::tmem_st16(t_s + c * 16, pk);
+            } else {
+                // no keys for this split: an empty partial (weight zero, but it is still read)
+                for (int e = 0; e < 128; e += 4) *reinterpret_cast<uint4 *>(dst + e) = make_uint4(0u, 0u, 0u, 0u);
             }
-            ptx::tmem_st_wait();
-            ptx::tc_fence_before();
-            ptx::mbar_arrive(bar(BAR_P + t));
+            park_ml[t * 128 + row] = make_float2(m_used, l);   // (-inf, 0) when this split had no keys
+            if (!ok) *abort_flag = 1;
         }
-        if (ok && !*abort_flag) ok = ptx::mbar_wait(bar(BAR_O + t), (cnt - 1) & 1);
-        if (ok && !*abort_flag) {
-            ptx::tc_fence_after();
-            float *dst = p.ws_o + (slab + t * 128 + row) * 128;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t o[32];
-                ptx::tmem_ld32(t_o + c * 32, o);
-                ptx::tmem_ld_wait();
-#pragma unroll
-                for (int e = 0; e < 32; e += 4)
-                    *reinterpret_cast<uint4 *>(dst + c * 32 + e) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
-            }
-            *reinterpret_cast<float2 *>(p.ws_ml + (slab + t * 128 + row) * 2) = make_float2(m_used, l);
-        }
-        if (!ok) *abort_flag = 1;
-    }
-
-    ptx::tc_fence_before();
-    __syncthreads();
-    if (*abort_flag) {
-        // A bounded wait ran out: raise the sticky error, give outstanding copies and tensor-core
-        // work one more bounded chance to finish, then release tensor memory.
-        if (threadIdx.x == 0) atomicExch(p.dev_error, MTV_ERR_TIMEOUT);
-        if (warp == 9 && lane == 0) {
-            ptx::mbar_wait(bar(BAR_Q), 0);
-            for (int s = 0; s < TC_SLOTS; ++s) { ptx::mbar_wait(bar(BAR_KV_FULL + s), 0); ptx::mbar_wait(bar(BAR_KV_FULL + s), 1); }
-        }
-        if (warp == 8) {
-            if (lane == 0) ptx::tc_commit(bar(BAR_FINAL));
-            __syncwarp();
-            ptx::mbar_wait(bar(BAR_FINAL), 0);
-        }
-        __syncthreads();
-    }
-    if (warp == 8) {
-        ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem, 512);
+        tc_epilogue<true>(p, ctx);
     }
 }
 
@@ -372,9 +651,44 @@ static bool encode_map(CUtensorMap *map, const void *base, const cuuint64_t dims
 
 bool attn_tc_eligible(int D, int G) { return D == 128 && (G == 1 || G == 2 || G == 4 || G == 8); }
 
+static int tc_prepare() {
+    static bool done = false;
+    if (!done) {
+        MTV_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
+        // the register rebalancing inside the kernel assumes the pool of a 168-register launch
+        cudaFuncAttributes fa;
+        MTV_CUDA_CHECK(cudaFuncGetAttributes(&fa, tree_attn_tc_kernel));
+        if (fa.numRegs < TC_REGS_LAUNCH) {
+            set_last_error("tree_attn_tc_kernel was built with too few registers for its setmaxnreg targets", cudaErrorInvalidValue);
+            return MTV_ERR_CUDA;
+        }
+        done = true;
+    }
+    return MTV_OK;
+}
+
+// Number of key splits of a problem: as many as keep the whole grid within one wave of SMs
+// (one CTA per SM), at most one per key tile, at most TC_MAX_SPLITS.  More than one split needs
+// a merge counter per query block.
+int attn_tc_plan(int T, int G, int B, int Hkv, int Lcap, int *n_rt_out) {
+    const int n_rt = (T * G + 255) / 256;
+    const long base = (long)B * Hkv * n_rt;
+    const int tiles = (Lcap + TC_BN - 1) / TC_BN;
+    long ns = sm_count() / base;
+    if (ns > tiles) ns = tiles;
+    if (ns > TC_MAX_SPLITS) ns = TC_MAX_SPLITS;
+#ifdef TC_FORCE_NSPLIT
+    ns = TC_FORCE_NSPLIT;
+#endif
+    if (ns < 1 || base > TC_MAX_GROUPS) ns = 1;
+    if (n_rt_out) *n_rt_out = n_rt;
+    return (int)ns;
+}
+
 int launch_tree_attn_tc(const mtv_tree *tree, int B, int Hq, int Hkv, const __nv_bfloat16 *q, const __nv_bfloat16 *k,
                         const __nv_bfloat16 *v, int64_t sb, int64_t sh, int64_t st, int Lcap, const int32_t *seq_lens,
-                        float scale_log2, float *ws_o, float *ws_ml, int nsplit, int m_rows, cudaStream_t stream) {
+                        float scale_log2, __nv_bfloat16 *out, int32_t *status, float *ws_o, float *ws_ml,
+                        cudaStream_t stream) {
     const int G = Hq / Hkv, T = tree->T, D = 128;
     CUtensorMap q_map, k_map, v_map;
     {
@@ -389,19 +703,32 @@ int launch_tree_attn_tc(const mtv_tree *tree, int B, int Hq, int Hkv, const __nv
         const cuuint32_t box[4] = {64, 128, 1, 1};
         if (!encode_map(&k_map, k, dims, str, box) || !encode_map(&v_map, v, dims, str, box)) return MTV_ERR_CUDA;
     }
-    static bool attr_done = false;
-    if (!attr_done) {
-        MTV_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
-        attr_done = true;
-    }
+    if (tc_prepare() != MTV_OK) return MTV_ERR_CUDA;
     TcParams p;
-    p.seq_lens = seq_lens; p.anc = tree->d_anc; p.ws_o = ws_o; p.ws_ml = ws_ml; p.dev_error = tree->d_error;
+    p.seq_lens = seq_lens; p.anc = tree->d_anc; p.out = out; p.status = status; p.dev_error = tree->d_error;
+    p.ws_o = ws_o; p.ws_ml = reinterpret_cast<float2 *>(ws_ml);
+    p.arrive = tree->d_counters; p.depart = tree->d_counters + TC_MAX_GROUPS;
     p.scale_log2 = scale_log2;
-    p.T = T; p.G = G; p.Hkv = Hkv; p.Lcap = Lcap; p.nsplit = nsplit; p.m_rows = m_rows; p.n_rt = m_rows / 256;
+    p.T = T; p.G = G; p.Hq = Hq; p.Hkv = Hkv; p.Lcap = Lcap;
+    p.nsplit = attn_tc_plan(T, G, B, Hkv, Lcap, &p.n_rt);
     p.M_rows = T * G;
-    const dim3 grid(nsplit, Hkv * p.n_rt, B);
-    tree_attn_tc_kernel<<<grid, TC_THREADS, TC_SMEM_BYTES, stream>>>(q_map, k_map, v_map, p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.nsplit, Hkv * p.n_rt, B);
+    cfg.blockDim = dim3(TC_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = TC_SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;   // CTAs that wait for each other must all be resident
+    attr[0].val.cooperative = p.nsplit > 1 ? 1 : 0;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    MTV_CUDA_CHECK(cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel, q_map, k_map, v_map, p));
     return MTV_OK;
 }
 
 }  // namespace mtv
+
+#ifdef MTV_TRACE
+extern "C" int mtv_trace_set(long long *buf) {
+    return cudaMemcpyToSymbol(mtv::g_trace, &buf, sizeof buf) == cudaSuccess ? 0 : -1;
+}
+#endif

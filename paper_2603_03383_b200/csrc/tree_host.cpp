@@ -136,7 +136,7 @@ extern "C" int tree_build_static(int K, int n_nodes, const int32_t *node_ranks, 
     if (upload) {
         const size_t n_ti = T, n_ri = (size_t)tr->P * (K + 1), n_anc = (size_t)T * 2;
         size_t o_ti = 0, o_ri = mtv::align_up(o_ti + n_ti * 4, 16), o_anc = mtv::align_up(o_ri + n_ri * 4, 16);
-        size_t o_kd = o_anc + n_anc * 8, o_co = o_kd + MTV_MAX_K * 4, o_err = o_co + MTV_MAX_K * 4, total = o_err + 16;
+        size_t o_kd = o_anc + n_anc * 8, o_co = o_kd + MTV_MAX_K * 4, o_err = o_co + MTV_MAX_K * 4, o_cnt = o_err + 16, total = o_cnt + 512 * 4;
         std::vector<unsigned char> blob(total, 0);
         memcpy(blob.data() + o_ti, tr->tree_indices.data(), n_ti * 4);
         memcpy(blob.data() + o_ri, tr->retrieve.data(), n_ri * 4);
@@ -161,6 +161,7 @@ extern "C" int tree_build_static(int K, int n_nodes, const int32_t *node_ranks, 
         tr->d_kd = (const int32_t *)(base + o_kd);
         tr->d_cand_offset = (const int32_t *)(base + o_co);
         tr->d_error = (int32_t *)(base + o_err);
+        tr->d_counters = (int32_t *)(base + o_cnt);
         tr->on_device = true;
     }
     *out = tr;
@@ -176,7 +177,10 @@ extern "C" void tree_destroy(mtv_tree_t *tree) {
 extern "C" int mtv_device_error(const mtv_tree_t *tree, int clear, int32_t *code) {
     if (!tree || !tree->on_device || !code) return MTV_ERR_INVALID_ARG;
     MTV_CUDA_CHECK(cudaMemcpy(code, tree->d_error, sizeof(int32_t), cudaMemcpyDeviceToHost));
-    if (clear && *code != 0) MTV_CUDA_CHECK(cudaMemset(tree->d_error, 0, sizeof(int32_t)));
+    if (clear && *code != 0) {   // an aborted kernel may also have left the merge counters dirty
+        MTV_CUDA_CHECK(cudaMemset(tree->d_error, 0, sizeof(int32_t)));
+        MTV_CUDA_CHECK(cudaMemset(tree->d_counters, 0, 512 * sizeof(int32_t)));
+    }
     return MTV_OK;
 }
 

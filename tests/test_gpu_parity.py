@@ -127,6 +127,25 @@ def test_attention_capacity_is_reported_not_faulted():
     assert_close(out[1:], want)
 
 
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 128), (8, 2, 64)])
+def test_attention_never_reads_past_the_tree_rows(Hq, Hkv, D):
+    """Cache rows behind the tree rows are uninitialised memory in real use: NaN there must not leak."""
+    tb, tree = make_tree("rank_prior", 4, (), 64)
+    T, B, Lcap = tree.T, 2, 400
+    lens = [200, 77]
+    q, k, v = synth.attention_inputs(B, T, Hq, Hkv, D, Lcap, 21)
+    sl = torch.tensor(lens, dtype=torch.int32)
+    want = ref.tree_attention(q, k, v, sl, tb["mask"])
+    kd, vd = k.to(DEV), v.to(DEV)
+    for b, L in enumerate(lens):
+        kd[b, :, L + T:] = float("nan")
+        vd[b, :, L + T:] = float("nan")
+    out = torch.zeros(B, T, Hq, D, dtype=torch.bfloat16, device=DEV)
+    ws = workspace(tree, B, 0, 0, Hq, Hkv, D, Lcap)
+    binding.tree_verify_attention(tree, q.to(DEV), kd, vd, sl.to(DEV), out, ws)
+    assert_close(out, want)
+
+
 def test_attention_explicit_scale():
     tb, tree = make_tree("cartesian", 2, (2, 2))
     T, D = tree.T, 64
