@@ -15,9 +15,10 @@
 // thread holds its whole row of S.
 //
 // The key splits of one query block are merged inside the same launch.  After its last key tile
-// a CTA parks its unnormalised partial (m, l, O) in shared memory, copies it coalesced to the
-// workspace (it stays in L2), and arrives on a counter of its query block.  When all splits of
-// the block have arrived, every CTA merges a slice of the rows from all partials, normalises
+// a CTA parks its unnormalised partial (m, l, O) in shared memory, sends it to the workspace with
+// bulk copies (it stays in L2), and arrives on a counter of its query block.  When all splits of
+// the block have arrived, every CTA fetches a slice of the rows of all partials with bulk copies
+// (plain loads would be throttled by the little L1 this kernel leaves), merges them, normalises
 // and writes bf16 output rows.  The launch is cooperative, so all CTAs are resident together and
 // the wait on the counter always ends; it is bounded all the same.  The counters live in the
 // tree object, start at zero and are put back to zero by the last CTA to leave.
@@ -34,7 +35,6 @@ namespace mtv {
 constexpr int TC_BN = 128;
 constexpr int TC_SLOTS = 5;
 constexpr int TC_THREADS = 384;   // 3 warpgroups: softmax 0, softmax 1, {MMA warp, TMA warp, 2 helper warps}
-constexpr int TC_SOFTMAX_THREADS = 256;
 constexpr uint32_t TC_TILE_BYTES = 128 * 128 * 2;   // one 128 x 128 bf16 tile: two 64-column halves
 constexpr uint32_t TC_HALF_BYTES = TC_TILE_BYTES / 2;
 constexpr uint32_t TC_Q_BYTES = 2 * TC_TILE_BYTES;
@@ -54,21 +54,26 @@ static_assert(2 * TC_REGS_SOFTMAX + TC_REGS_OTHER <= 3 * TC_REGS_LAUNCH, "setmax
 static_assert(TC_REGS_LAUNCH * TC_THREADS <= 65536, "launch register count does not fit the register file");
 
 // After the last key tile the Q / K / V buffers are reused:
-//   [0, PARK_O)            parked O, 256 rows of TC_O_STRIDE floats (528 bytes: conflict-free 16-byte stores)
-//   [PARK_O, +2048)        parked (m, l) per row
-//   [.., +WBUF)            (m, l) of every split for the rows this CTA merges, then their weights
-//   [.., +1024)            1 / l of the merged rows
-constexpr int TC_O_STRIDE = 132;
-constexpr uint32_t TC_PARK_O_BYTES = 256 * TC_O_STRIDE * 4;
-constexpr uint32_t TC_PARK_ML_OFF = TC_PARK_O_BYTES;
+//   [0, 128 KB)      the parked partial O: 256 rows of 512 bytes; 16-byte chunk j of row r sits at
+//                    chunk position j ^ (r & 31), which makes the one-row-per-thread stores
+//                    conflict-free while rows stay contiguous for one bulk copy.  The workspace
+//                    holds partials in the same form; whoever reads a row undoes the permutation.
+//                    After the partial has left for the workspace the same space receives the
+//                    rows this CTA merges, from all splits.
+//   the last 8 KB    parked (m, l) per row; (m, l) then weights of every split for the merged
+//                    rows; 1 / l of the merged rows
+constexpr uint32_t TC_ROW_BYTES = 512;
+constexpr uint32_t TC_TILES_BYTES = TC_Q_BYTES + TC_RING_BYTES;
+constexpr uint32_t TC_PARK_ML_OFF = TC_TILES_BYTES - 8192;
 constexpr uint32_t TC_WBUF_OFF = TC_PARK_ML_OFF + 256 * 8;
 constexpr uint32_t TC_WBUF_ENTRIES = 256 + TC_MAX_SPLITS;
 constexpr uint32_t TC_ROWINV_OFF = TC_WBUF_OFF + TC_WBUF_ENTRIES * 8;
-static_assert(TC_ROWINV_OFF + 256 * 4 <= TC_Q_BYTES + TC_RING_BYTES, "merge buffers must fit the tile buffers");
+static_assert(TC_ROWINV_OFF + 256 * 4 <= TC_TILES_BYTES, "merge buffers must fit the tile buffers");
+static_assert((256 + TC_MAX_SPLITS) * TC_ROW_BYTES <= TC_PARK_ML_OFF, "rows to merge must fit below the small buffers");
 
 // barrier slots (8 bytes each) inside the barrier region
 enum { BAR_Q = 0, BAR_KV_FULL = 1, BAR_KV_EMPTY = BAR_KV_FULL + TC_SLOTS, BAR_S = BAR_KV_EMPTY + TC_SLOTS,
-       BAR_P = BAR_S + 2, BAR_O = BAR_P + 2, BAR_FINAL = BAR_O + 2, BAR_COUNT = BAR_FINAL + 1 };
+       BAR_P = BAR_S + 2, BAR_O = BAR_P + 2, BAR_FINAL = BAR_O + 2, BAR_MERGE = BAR_FINAL + 1, BAR_COUNT = BAR_MERGE + 1 };
 static_assert(BAR_COUNT * 8 + 8 <= TC_BAR_BYTES, "barrier region too small");
 
 // instruction descriptors: bf16 x bf16 -> fp32, M = 128, N = 128
@@ -80,7 +85,7 @@ struct TcParams {
     const int32_t *seq_lens;
     const uint64_t *anc;   // [T][2]
     __nv_bfloat16 *out;    // [B][T][Hq][128]
-    float *ws_o;           // [groups][nsplit][256][128] partial O (only when nsplit > 1)
+    float *ws_o;           // [groups][nsplit][256 rows][128] partial O, chunks permuted (only when nsplit > 1)
     float2 *ws_ml;         // [groups][nsplit][256] partial (m, l)
     int32_t *arrive, *depart;   // [groups] merge counters, zero between calls
     int32_t *status;       // [B] or null
@@ -155,7 +160,6 @@ struct TcCtx {
 template <bool SOFTMAX>
 __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    float *park_o = reinterpret_cast<float *>(c.tiles);
     float2 *park_ml = reinterpret_cast<float2 *>(c.tiles + TC_PARK_ML_OFF);
     float2 *wbuf = reinterpret_cast<float2 *>(c.tiles + TC_WBUF_OFF);
     float *rowinv = reinterpret_cast<float *>(c.tiles + TC_ROWINV_OFF);
@@ -186,12 +190,17 @@ __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
     const int act_rows = c.nt * 128;
     const int nsplit = p.nsplit;
     const int grp = blockIdx.z * gridDim.y + blockIdx.y;
+    const unsigned char *rows_smem = c.tiles;   // parked rows, later the rows to merge
+    // chunk j (16 bytes) of a 512-byte row whose index inside its 256-row slab is r
+    auto chunk = [&](const unsigned char *row_ptr, int r, int j) {
+        return *reinterpret_cast<const float4 *>(row_ptr + ((j ^ (r & 31)) << 4));
+    };
     if (nsplit == 1) {
         // the partial is the result: normalise and store
         for (int item = threadIdx.x; item < act_rows * 32; item += TC_THREADS) {
             const int row = item / 32, c4 = item % 32, r = c.rows0 + row;
             if (r >= p.M_rows) continue;
-            const float4 v = *reinterpret_cast<const float4 *>(park_o + row * TC_O_STRIDE + c4 * 4);
+            const float4 v = chunk(rows_smem + row * TC_ROW_BYTES, row, c4);
             const float inv = 1.f / park_ml[row].y;
             uint2 packed;
             packed.x = pack2_bf16(v.x * inv, v.y * inv);
@@ -200,98 +209,71 @@ __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
             *reinterpret_cast<uint2 *>(p.out + (((size_t)c.b * p.T + node) * p.Hq + hq) * 128 + c4 * 4) = packed;
         }
     } else {
-        // ---- publish the partial
-        const size_t slab = ((size_t)grp * nsplit + c.split) * 256;
-        for (int idx = threadIdx.x; idx < act_rows * 32; idx += TC_THREADS) {
-            const int row = idx / 32, c4 = idx % 32;
-            *reinterpret_cast<float4 *>(p.ws_o + (slab + row) * 128 + c4 * 4) =
-                *reinterpret_cast<const float4 *>(park_o + row * TC_O_STRIDE + c4 * 4);
-        }
-        for (int row = threadIdx.x; row < act_rows; row += TC_THREADS) p.ws_ml[slab + row] = park_ml[row];
-        cta_sync();
+        const size_t slab0 = (size_t)grp * nsplit;   // first slab of this query block
+        const int rows_per = (act_rows + nsplit - 1) / nsplit;
+        const int row_begin = c.split * rows_per;
+        const int n_my = max(0, min(act_rows, row_begin + rows_per) - row_begin);
         if (threadIdx.x == 0) {
-            __threadfence();   // cumulative: covers the CTA's stores ordered before the barrier
+            // ---- publish: two bulk copies out of shared memory, then arrive and wait for the others
+            const size_t slab = slab0 + c.split;
+            ptx::bulk_s2g(p.ws_o + slab * 256 * 128, ptx::smem_u32(c.tiles), act_rows * TC_ROW_BYTES);
+            ptx::bulk_s2g(p.ws_ml + slab * 256, ptx::smem_u32(c.tiles + TC_PARK_ML_OFF), act_rows * 8);
+            ptx::bulk_commit();
+            ptx::bulk_wait_all();
+            ptx::fence_proxy_async_all();
+            __threadfence();
             atomicAdd(p.arrive + grp, 1);
             const long long t0 = clock64();
             while (ld_acquire(p.arrive + grp) < nsplit)
                 if (clock64() - t0 > ptx::WAIT_CYCLE_LIMIT) { atomicExch(p.dev_error, MTV_ERR_TIMEOUT); break; }
+            ptx::fence_proxy_async_all();
+            // ---- fetch rows [row_begin, row_begin + n_my) of every split: one bulk copy per split
+            if (n_my > 0) {
+                ptx::mbar_arrive_expect_tx(bar(BAR_MERGE), (uint32_t)(nsplit * n_my) * TC_ROW_BYTES);
+                for (int sp = 0; sp < nsplit; ++sp)
+                    ptx::bulk_g2s(ptx::smem_u32(c.tiles) + (uint32_t)(sp * n_my) * TC_ROW_BYTES,
+                                  p.ws_o + ((slab0 + sp) * 256 + row_begin) * 128, (uint32_t)n_my * TC_ROW_BYTES, bar(BAR_MERGE));
+            }
         }
         cta_sync();
-        if (warp == 0) TRACE(45);   // all splits arrived
-
-        // ---- merge rows [row_begin, row_begin + n_my) of the query block from all splits
-        const int rows_per = (act_rows + nsplit - 1) / nsplit;
-        const int row_begin = c.split * rows_per;
-        const int n_my = max(0, min(act_rows, row_begin + rows_per) - row_begin);
-        const size_t src0 = (size_t)grp * nsplit * 256 + row_begin;   // + s * 256 + local row
+        if (warp == 0) TRACE(45);   // all splits arrived, rows on their way
         for (int idx = threadIdx.x; idx < n_my * nsplit; idx += TC_THREADS) {
-            const int rl = idx / nsplit, s = idx - rl * nsplit;
-            wbuf[idx] = __ldcg(p.ws_ml + src0 + (size_t)s * 256 + rl);
-        }
-        // Thread tid of the softmax warpgroups owns the items (row, 4 columns) tid, tid + 256, ...;
-        // its loads of all splits are independent of the weights, so they go out first.
-        constexpr int NBUF = 36;
-        float4 v[NBUF];
-        const int n_items = n_my * 32;
-        const int my_items = SOFTMAX && (int)threadIdx.x < n_items ? (n_items - (int)threadIdx.x + TC_SOFTMAX_THREADS - 1) / TC_SOFTMAX_THREADS : 0;
-        const int n_pairs = my_items * nsplit;     // pair q = k * nsplit + s: item k of this thread, split s
-        auto pair_src = [&](int q) {
-            const int k = q / nsplit, s = q - k * nsplit;
-            const int item = threadIdx.x + k * TC_SOFTMAX_THREADS;
-            return reinterpret_cast<const float4 *>(p.ws_o + (src0 + (size_t)s * 256 + item / 32) * 128 + (item % 32) * 4);
-        };
-        if (SOFTMAX) {
-#pragma unroll
-            for (int u = 0; u < NBUF; ++u)
-                if (u < n_pairs) v[u] = __ldcg(pair_src(u));
+            const int rl = idx / nsplit, sp = idx - rl * nsplit;
+            wbuf[idx] = __ldcg(p.ws_ml + (slab0 + sp) * 256 + row_begin + rl);
         }
         cta_sync();
         for (int rl = threadIdx.x; rl < n_my; rl += TC_THREADS) {
             float m = -INFINITY;
-            for (int s = 0; s < nsplit; ++s) m = fmaxf(m, wbuf[rl * nsplit + s].x);
+            for (int sp = 0; sp < nsplit; ++sp) m = fmaxf(m, wbuf[rl * nsplit + sp].x);
             float lsum = 0.f;
-            for (int s = 0; s < nsplit; ++s) {
-                const float2 ml = wbuf[rl * nsplit + s];
+            for (int sp = 0; sp < nsplit; ++sp) {
+                const float2 ml = wbuf[rl * nsplit + sp];
                 const float w = ml.x == -INFINITY ? 0.f : ex2(ml.x - m);
                 lsum += w * ml.y;
-                wbuf[rl * nsplit + s].x = w;
+                wbuf[rl * nsplit + sp].x = w;
             }
             rowinv[rl] = 1.f / lsum;
         }
         cta_sync();
-        if (SOFTMAX) {
+        if (n_my > 0 && !ptx::mbar_wait(bar(BAR_MERGE), 0) && threadIdx.x == 0) atomicExch(p.dev_error, MTV_ERR_TIMEOUT);
+        for (int item = threadIdx.x; item < n_my * 32; item += TC_THREADS) {
+            const int rl = item / 32, c4 = item % 32;
+            const int r = c.rows0 + row_begin + rl;
+            if (r >= p.M_rows) continue;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int q0 = 0; q0 < n_pairs; q0 += NBUF) {
-                if (q0 > 0) {
-#pragma unroll
-                    for (int u = 0; u < NBUF; ++u)
-                        if (q0 + u < n_pairs) v[u] = __ldcg(pair_src(q0 + u));
-                }
-#pragma unroll
-                for (int u = 0; u < NBUF; ++u) {
-                    const int q = q0 + u;
-                    if (q < n_pairs) {
-                        const int k = q / nsplit, s = q - k * nsplit;
-                        const int item = threadIdx.x + k * TC_SOFTMAX_THREADS;
-                        const int rl = item / 32, c4 = item % 32;
-                        const float w = wbuf[rl * nsplit + s].x;
-                        acc.x = fmaf(w, v[u].x, acc.x); acc.y = fmaf(w, v[u].y, acc.y);
-                        acc.z = fmaf(w, v[u].z, acc.z); acc.w = fmaf(w, v[u].w, acc.w);
-                        if (s == nsplit - 1) {
-                            const int r = c.rows0 + row_begin + rl;
-                            if (r < p.M_rows) {
-                                const float inv = rowinv[rl];
-                                uint2 packed;
-                                packed.x = pack2_bf16(acc.x * inv, acc.y * inv);
-                                packed.y = pack2_bf16(acc.z * inv, acc.w * inv);
-                                const int node = r / p.G, hq = c.g * p.G + r % p.G;
-                                *reinterpret_cast<uint2 *>(p.out + (((size_t)c.b * p.T + node) * p.Hq + hq) * 128 + c4 * 4) = packed;
-                            }
-                            acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                        }
-                    }
-                }
+            const unsigned char *row_ptr = rows_smem + rl * TC_ROW_BYTES;
+            for (int sp = 0; sp < nsplit; ++sp) {
+                const float w = wbuf[rl * nsplit + sp].x;
+                const float4 v = chunk(row_ptr + (size_t)(sp * n_my) * TC_ROW_BYTES, row_begin + rl, c4);
+                acc.x = fmaf(w, v.x, acc.x); acc.y = fmaf(w, v.y, acc.y);
+                acc.z = fmaf(w, v.z, acc.z); acc.w = fmaf(w, v.w, acc.w);
             }
+            const float inv = rowinv[rl];
+            uint2 packed;
+            packed.x = pack2_bf16(acc.x * inv, acc.y * inv);
+            packed.y = pack2_bf16(acc.z * inv, acc.w * inv);
+            const int node = r / p.G, hq = c.g * p.G + r % p.G;
+            *reinterpret_cast<uint2 *>(p.out + (((size_t)c.b * p.T + node) * p.Hq + hq) * 128 + c4 * 4) = packed;
         }
         if (warp == 0) TRACE(46);   // merge done
         // the last CTA of the query block to get here puts the counters back to zero
@@ -343,7 +325,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(bar_region + BAR_COUNT * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bar_region + BAR_COUNT * 8 + 4);
     auto bar = [&](int i) { return bars + (uint32_t)i * 8u; };
-    float *park_o = reinterpret_cast<float *>(tiles_gen);
     float2 *park_ml = reinterpret_cast<float2 *>(tiles_gen + TC_PARK_ML_OFF);
 
     // One K or V tile into ring slot (i mod TC_SLOTS): i = 2j is K of key tile j, i = 2j + 1 is V.
@@ -367,6 +348,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
             ptx::mbar_init(bar(BAR_O + t), 1);
         }
         ptx::mbar_init(bar(BAR_FINAL), 1);
+        ptx::mbar_init(bar(BAR_MERGE), 1);
         ptx::fence_mbar_init();
         *abort_flag = 0;
         if (cnt > 0) {
@@ -592,29 +574,35 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
                 ptx::mbar_arrive(bar(BAR_P + t));
                 if (warp % 4 == 0 && j < 6) TRACE(9 + t * 16 + j * 2);       // P_t(j) written
             }
-            // ---- park the partial of this row in shared memory
-            float *dst = park_o + (t * 128 + row) * TC_O_STRIDE;
+            // ---- hand over the partial of this row
             if (cnt > 0) {
                 // every tensor-core read of the tile buffers must be over before they are reused
                 if (ok && !*abort_flag) ok = ptx::mbar_wait(bar(BAR_FINAL), 0);
                 if (warp % 4 == 0) TRACE(40 + t);                            // all tensor-core work done
-                if (ok && !*abort_flag) {
-                    ptx::tc_fence_after();
+                if (ok) ptx::tc_fence_after();
+            }
+            const bool have_o = cnt > 0 && ok && !*abort_flag;
+            {
+                // park the row: chunk j at position j ^ (row & 31); an empty split parks zeros
+                unsigned char *dst = tiles_gen + (t * 128 + row) * TC_ROW_BYTES;
+                const int sw = (t * 128 + row) & 31;
 #pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t o[32];
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t o[32];
+                    if (have_o) {
                         ptx::tmem_ld32(t_o + c * 32, o);
                         ptx::tmem_ld_wait();
+                    } else {
 #pragma unroll
-                        for (int e = 0; e < 32; e += 4)
-                            *reinterpret_cast<uint4 *>(dst + c * 32 + e) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
+                        for (int e = 0; e < 32; ++e) o[e] = 0u;
                     }
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4)
+                        *reinterpret_cast<uint4 *>(dst + (((c * 8 + e / 4) ^ sw) << 4)) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
                 }
-            } else {
-                // no keys for this split: an empty partial (weight zero, but it is still read)
-                for (int e = 0; e < 128; e += 4) *reinterpret_cast<uint4 *>(dst + e) = make_uint4(0u, 0u, 0u, 0u);
+                park_ml[t * 128 + row] = make_float2(m_used, l);   // (-inf, 0) for an empty split
+                ptx::fence_proxy_async();   // the bulk copy out of shared memory must see these stores
             }
-            park_ml[t * 128 + row] = make_float2(m_used, l);   // (-inf, 0) when this split had no keys
             if (!ok) *abort_flag = 1;
         }
         tc_epilogue<true>(p, ctx);
