@@ -107,7 +107,23 @@ class ClockSampler:
                     reasons=sorted(reasons), samples=len(sm))
 
 
-def build_problem(w, n_layers, device):
+def rank_seed(w, rank):
+    """Seed of the sequences rank `rank` verifies (ranks work on independent sequences)."""
+    return w.seed + 7919 * rank
+
+
+def max_over_ranks(value, world, device=None):
+    """Largest `value` over all ranks (the job is as slow as its slowest rank)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.item()
+
+
+def build_problem(w, n_layers, device, seed=None):
     """Everything one rank needs, resident on `device`.  Returns a dict."""
     import torch
     from paper_2603_03383_b200 import binding, synth
@@ -115,9 +131,10 @@ def build_problem(w, n_layers, device):
              else binding.tree_gen_rank_prior(w.K, w.T, w.R_max))
     tree = binding.tree_build_static(w.K, nodes, upload=True)
     T, B = tree.T, w.B
-    lens = synth.seq_lens(w)
+    seed = w.seed if seed is None else seed
+    lens = synth.seq_lens(w, seed=seed)
     Lcap = int(w.L_hi) + T
-    seed = w.seed
+    seed = w.seed if seed is None else seed
     hidden, W1, b1, W2, root = synth.head_inputs(B, w.H, w.V, w.K, seed, device=device)
     ws = torch.empty(binding.mtv_workspace_bytes(tree, B, w.H, w.V, w.Hq, w.Hkv, w.D, Lcap), dtype=torch.uint8,
                      device=device)
@@ -169,7 +186,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
     w = synth.WORKLOADS[args.workload]
     n_layers = args.layers
-    P = build_problem(w, n_layers, dev)
+    P = build_problem(w, n_layers, dev, seed=rank_seed(w, rank))
     tree, a = P["tree"], P["args"]
     K_steps, W_steps = args.steps, max(args.warmup, 3)
 
@@ -202,10 +219,7 @@ def run_ours(args):
         taps.__exit__()
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = t.item()
+    ms_total = max_over_ranks(ms_total, world, dev)
     ms_step = ms_total / K_steps
     value = world * 1000.0 / ms_step
     mean_tokens = (P["accept_len"].float().mean().item() + 1.0)
@@ -230,10 +244,7 @@ def run_ours(args):
         binding.mtv_verify_step_host(tree, a, hb)
     torch.cuda.synchronize()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_s], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = t.item()
+    e2e_s = max_over_ranks(e2e_s, world, dev)
 
     if rank != 0:
         if world > 1:
