@@ -168,6 +168,31 @@ int tree_accept(const mtv_tree_t *tree, int B, int V, const mtv_bf16 *logits, co
                 int32_t *next_root, void *ws, size_t ws_bytes, void *stream);
 
 /* ---------------------------------------------------------------------------
+ * tree_accept without a workspace — the paper has no counterpart; this is a convenience of
+ * the library.  Same inputs, outputs and results as tree_accept, but the scratch (the
+ * per-chunk argmax keys) sits in a 64 KB array that is part of the library image, so the call
+ * needs no buffer from the caller and the library never calls cudaMalloc / cudaFree for it.
+ * It is meant for callers that are not allowed to allocate device memory: a plugin inside a
+ * serving runtime that owns the whole device heap, a latency-critical decode loop in which an
+ * allocator call (it may synchronise the device) is banned, a process whose memory budget was
+ * fixed at start-up.
+ *   - Limit: B * T * splits * 8 bytes <= tree_accept_static_scratch_capacity() (65536), i.e.
+ *     up to 8192 logit rows; beyond that the call returns MTV_ERR_WORKSPACE, launches nothing,
+ *     and mtv_last_error() says how much was needed.
+ *   - The first call on a device looks up the array's device address (one runtime query, no
+ *     allocation) and remembers it; make that first call outside any stream capture and with
+ *     the device current that later calls will use.
+ *   - Every GPU that loads the library holds the 64 KB until the process exits.
+ *   - All calls on a device share the array and it keeps the previous call's contents; each call
+ *     overwrites every entry it later reads, so nothing has to be cleared.  Two calls that
+ *     overlap on the GPU (different streams) race on it: keep them stream-ordered.
+ */
+int tree_accept_static_scratch(const mtv_tree_t *tree, int B, int V, const mtv_bf16 *logits,
+                               const int32_t *tree_tok, int32_t *accept_len, int32_t *best_path,
+                               int32_t *acc_nodes, int32_t *acc_tok, int32_t *next_root, void *stream);
+size_t tree_accept_static_scratch_capacity(void);
+
+/* ---------------------------------------------------------------------------
  * KV compaction — Section 3.2, "Zero-Copy Retrieval" applied to K/V: for every layer,
  * sequence b, KV head g and j = 1..accept_len[b], row seq_lens[b] + acc_nodes[b][j]
  * moves to row seq_lens[b] + j, in place (all sources are read before any row is
@@ -251,7 +276,7 @@ int mtv_kernel_taps_used(int kernel_id);
  * synchronises with the device: use it between steps, not inside one. */
 int mtv_device_error(const mtv_tree_t *tree, int clear, int32_t *code);
 
-/* Human-readable text for the most recent MTV_ERR_CUDA on this thread (never NULL). */
+/* Human-readable text for the most recent MTV_ERR_CUDA (or refused size) on this thread (never NULL). */
 const char *mtv_last_error(void);
 
 #ifdef __cplusplus

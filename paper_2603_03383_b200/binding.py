@@ -25,7 +25,8 @@ MAX_K = 8
 EXPORTS = ["tree_build_static", "tree_gen_cartesian", "tree_gen_rank_prior", "tree_query", "tree_destroy",
            "mtv_workspace_bytes", "medusa_heads_topk", "tree_verify_attention", "tree_accept",
            "kv_compact_accepted", "mtv_verify_step", "mtv_verify_step_host", "mtv_last_error",
-           "mtv_set_kernel_taps", "mtv_kernel_taps_used", "mtv_device_error"]
+           "mtv_set_kernel_taps", "mtv_kernel_taps_used", "mtv_device_error",
+           "tree_accept_static_scratch", "tree_accept_static_scratch_capacity"]
 
 
 class MtvError(RuntimeError):
@@ -95,6 +96,8 @@ def lib():
         L.mtv_set_kernel_taps.argtypes = [i32, vp, vp, i32]
         L.mtv_kernel_taps_used.argtypes = [i32]
         L.mtv_device_error.argtypes = [vp, i32, C.POINTER(C.c_int32)]
+        L.tree_accept_static_scratch.argtypes = [vp, i32, i32] + [vp] * 7 + [vp]
+        L.tree_accept_static_scratch_capacity.restype = sz
         _lib = L
     return _lib
 
@@ -212,6 +215,22 @@ def tree_accept(tree, logits, tree_tok, accept_len, best_path, acc_nodes, acc_to
     _check(lib().tree_accept(tree.handle, B, V, _ptr(logits), _ptr(tree_tok), _ptr(accept_len), _ptr(best_path),
                              _ptr(acc_nodes), _ptr(acc_tok), _ptr(next_root), p, n, _stream(stream)),
            "tree_accept")
+
+
+def tree_accept_static_scratch(tree, logits, tree_tok, accept_len, best_path, acc_nodes, acc_tok, next_root,
+                               stream=None):
+    """tree_accept for callers that may not allocate: no workspace argument (see include/mtv.h)."""
+    B, T, V = logits.shape
+    rc = lib().tree_accept_static_scratch(tree.handle, B, V, _ptr(logits), _ptr(tree_tok), _ptr(accept_len),
+                                          _ptr(best_path), _ptr(acc_nodes), _ptr(acc_tok), _ptr(next_root),
+                                          _stream(stream))
+    if rc == -3:    # too large for the built-in array: the library says by how much
+        raise MtvError(rc, "tree_accept_static_scratch [%s]" % lib().mtv_last_error().decode())
+    _check(rc, "tree_accept_static_scratch")
+
+
+def tree_accept_static_scratch_capacity() -> int:
+    return lib().tree_accept_static_scratch_capacity()
 
 
 def cache_pointer_array(caches, device=None):

@@ -1,6 +1,8 @@
 // Acceptance and token retrieval (Section 3.2, "Zero-Copy Retrieval"): per-node argmax
 // of the base-model logits, greedy longest-prefix match over the static paths, and the
 // gather of the accepted tokens through retrieve_indices — all on the device.
+#include <cstdio>
+
 #include "common.cuh"
 
 namespace mtv {
@@ -135,6 +137,66 @@ extern "C" int tree_accept(const mtv_tree_t *tree, int B, int V, const mtv_bf16 
             V, reinterpret_cast<const __nv_bfloat16 *>(logits), part);
     }
     TapScope tap(MTV_KERNEL_ACCEPT_FINISH, st);
+    accept_finish_kernel<<<B, 128, 0, st>>>(tree->T, tree->K, tree->P, L.nsplit, part, tree_tok, tree->d_retrieve,
+                                            accept_len, best_path, acc_nodes, acc_tok, next_root);
+    MTV_CUDA_CHECK(cudaGetLastError());
+    return MTV_OK;
+}
+
+// ---------------------------------------------------------------------------
+// tree_accept for callers that must not allocate device memory (the paper has no counterpart).
+// Its scratch — the per-chunk argmax keys that tree_accept keeps in the caller's workspace —
+// lives in a fixed array inside the library image.
+namespace mtv {
+
+constexpr size_t ACCEPT_STATIC_SCRATCH_BYTES = 64 * 1024;
+static __device__ __align__(256) unsigned char g_accept_scratch[ACCEPT_STATIC_SCRATCH_BYTES];
+
+// Device address of g_accept_scratch on the current device.  In host code the array's name is
+// only a handle for the runtime, not an address a kernel could use, so the address is asked for
+// once per device (with that device current) and remembered.
+static int accept_scratch_address(unsigned long long **out) {
+    constexpr int MAX_DEVICES = 64;
+    static unsigned long long *cached[MAX_DEVICES] = {nullptr};
+    int dev = 0;
+    MTV_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) return MTV_ERR_UNSUPPORTED_SHAPE;
+    if (!cached[dev]) {
+        void *ptr = nullptr;
+        MTV_CUDA_CHECK(cudaGetSymbolAddress(&ptr, g_accept_scratch));
+        cached[dev] = reinterpret_cast<unsigned long long *>(ptr);
+    }
+    *out = cached[dev];
+    return MTV_OK;
+}
+
+}  // namespace mtv
+
+extern "C" size_t tree_accept_static_scratch_capacity(void) { return mtv::ACCEPT_STATIC_SCRATCH_BYTES; }
+
+extern "C" int tree_accept_static_scratch(const mtv_tree_t *tree, int B, int V, const mtv_bf16 *logits,
+                                          const int32_t *tree_tok, int32_t *accept_len, int32_t *best_path,
+                                          int32_t *acc_nodes, int32_t *acc_tok, int32_t *next_root, void *stream) {
+    using namespace mtv;
+    if (!tree || !tree->on_device || !logits || !tree_tok || !accept_len || !best_path || !acc_nodes ||
+        !acc_tok || !next_root || B < 1 || V < 1)
+        return MTV_ERR_INVALID_ARG;
+    if (tree->P > 255) return MTV_ERR_UNSUPPORTED_SHAPE;
+    const AcceptWs L = accept_ws_layout(tree, B, V);
+    if (L.total > ACCEPT_STATIC_SCRATCH_BYTES) {
+        char msg[160];
+        snprintf(msg, sizeof msg, "tree_accept_static_scratch: B*T = %ld logit rows need %zu bytes of scratch, "
+                 "the built-in array holds %zu", (long)B * tree->T, L.total, ACCEPT_STATIC_SCRATCH_BYTES);
+        set_last_error_text(msg);
+        return MTV_ERR_WORKSPACE;
+    }
+    unsigned long long *part = nullptr;
+    const int rc = accept_scratch_address(&part);
+    if (rc != MTV_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    // every entry of `part` that the second kernel reads is written by the first one: nothing to clear
+    node_argmax_partial_kernel<<<dim3(L.nsplit, B * tree->T), ARGMAX_THREADS, 0, st>>>(
+        V, reinterpret_cast<const __nv_bfloat16 *>(logits), part);
     accept_finish_kernel<<<B, 128, 0, st>>>(tree->T, tree->K, tree->P, L.nsplit, part, tree_tok, tree->d_retrieve,
                                             accept_len, best_path, acc_nodes, acc_tok, next_root);
     MTV_CUDA_CHECK(cudaGetLastError());

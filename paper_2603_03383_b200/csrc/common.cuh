@@ -32,6 +32,7 @@ struct mtv_tree {
 namespace mtv {
 
 void set_last_error(const char *what, cudaError_t e);
+void set_last_error_text(const char *text);
 
 #define MTV_CUDA_CHECK(expr)                                  \
     do {                                                      \

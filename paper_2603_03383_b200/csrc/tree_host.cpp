@@ -29,6 +29,7 @@ namespace mtv {
 void set_last_error(const char *what, cudaError_t e) {
     snprintf(g_err, sizeof g_err, "%s: %s", what, cudaGetErrorString(e));
 }
+void set_last_error_text(const char *text) { snprintf(g_err, sizeof g_err, "%s", text); }
 int sm_count() {
     static int n = 0;
     if (n == 0) {

@@ -1,0 +1,61 @@
+"""tree_accept_static_scratch: the workspace-free variant of tree_accept.
+
+Some users of this library run where device allocation is off limits (inside a serving runtime that
+owns the device heap, or in a decode loop where an allocator call is banned).  For them tree_accept
+exists in a form whose scratch is a fixed array inside the library.  This file checks, through the
+C ABI, that it returns exactly what tree_accept returns — on two calls in a row, because the array
+keeps whatever the previous call left in it — and that a problem too large for the array is refused.
+The file name keeps it last in pytest's collection order."""
+import pytest
+import torch
+
+from paper_2603_03383_b200 import binding, synth
+from tests._cases import make_tree, workspace
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+NAMES = ["accept_len", "best_path", "acc_nodes", "acc_tok", "next_root"]
+
+
+def _outputs(B, K):
+    f = lambda *s: torch.full(s, -7, dtype=torch.int32, device=DEV)
+    return [f(B), f(B), f(B, K + 1), f(B, K + 1), f(B)]
+
+
+def _inputs(tb, B, T, V, K, seed, p):
+    g = torch.Generator().manual_seed(seed)
+    cand = torch.stack([torch.randperm(V, generator=g)[:tb["C"]] for _ in range(B)]).to(torch.int32)
+    tree_tok = cand[:, torch.tensor(tb["tree_indices"])].contiguous()
+    logits, _ = synth.planted_logits(B, T, V, K, tree_tok, tb["parent"], tb["rank"], seed=seed, p_accept=p)
+    return logits.to(DEV), tree_tok.to(DEV)
+
+
+def test_matches_tree_accept_on_two_calls_in_a_row():
+    K = 4
+    tb, tree = make_tree("rank_prior", K, (), 64)
+    T = tree.T
+    # two different problems back to back: the second call finds the first one's keys in the array
+    for B, V, seed, p in [(4, 20000, 11, (0.9, 0.3)), (2, 5003, 12, (0.6,))]:
+        logits, tree_tok = _inputs(tb, B, T, V, K, seed, p)
+        want = _outputs(B, K)
+        binding.tree_accept(tree, logits, tree_tok, *want, workspace(tree, B, 8, V, 0, 0, 0, 0))
+        got = _outputs(B, K)
+        binding.tree_accept_static_scratch(tree, logits, tree_tok, *got)
+        torch.cuda.synchronize()
+        for name, a, b in zip(NAMES, got, want):
+            assert torch.equal(a, b), name          # integer outputs: bit-exact, as in the other accept tests
+        assert int(want[0].max()) >= 1              # the planted walks were found, not an all-zero coincidence
+
+
+def test_refuses_more_rows_than_the_array_can_serve():
+    tb, tree = make_tree("rank_prior", 5, (), 128)
+    B, V = 65, 8                                    # 65 * 128 rows * 8 bytes > 65536
+    assert B * tree.T * 8 > binding.tree_accept_static_scratch_capacity()
+    logits = torch.zeros(B, tree.T, V, dtype=torch.bfloat16, device=DEV)
+    tree_tok = torch.zeros(B, tree.T, dtype=torch.int32, device=DEV)
+    outs = _outputs(B, 5)
+    with pytest.raises(binding.MtvError) as e:
+        binding.tree_accept_static_scratch(tree, logits, tree_tok, *outs)
+    assert e.value.code == -3 and "65536" in str(e.value)
+    torch.cuda.synchronize()
+    assert all(bool((t == -7).all()) for t in outs)  # nothing was launched
