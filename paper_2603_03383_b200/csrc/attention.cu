@@ -20,7 +20,7 @@ bool attn_tc_eligible(int D, int G);
 int attn_tc_plan(int T, int G, int B, int Hkv, int Lcap, int *n_rt_out);
 int launch_tree_attn_tc(const mtv_tree *tree, int B, int Hq, int Hkv, const __nv_bfloat16 *q, const __nv_bfloat16 *k,
                         const __nv_bfloat16 *v, int64_t sb, int64_t sh, int64_t st, int Lcap, const int32_t *seq_lens,
-                        float scale_log2, __nv_bfloat16 *out, int32_t *status, float *ws_o, float *ws_ml,
+                        float scale_log2, __nv_bfloat16 *out, int32_t *status, void *ws_o, float *ws_ml,
                         cudaStream_t stream);
 
 AttnWs attn_ws_layout(const mtv_tree *t, int B, int Hq, int Hkv, int D, int Lcap) {
@@ -34,7 +34,7 @@ AttnWs attn_ws_layout(const mtv_tree *t, int B, int Hq, int Hkv, int D, int Lcap
         w.m_rows = 256;
         const size_t slabs = w.nsplit > 1 ? (size_t)B * Hkv * n_rt * w.nsplit : 0;
         w.o_off = 0;
-        w.ml_off = align_up(slabs * 256 * D * sizeof(float), 256);
+        w.ml_off = align_up(slabs * 256 * D * sizeof(__nv_bfloat16), 256);
         w.total = align_up(w.ml_off + slabs * 256 * 2 * sizeof(float), 256) + 256;
         return w;
     }

@@ -15,11 +15,13 @@
 // thread holds its whole row of S.
 //
 // The key splits of one query block are merged inside the same launch.  After its last key tile
-// a CTA parks its unnormalised partial (m, l, O) in shared memory, sends it to the workspace with
-// bulk copies (it stays in L2), and arrives on a counter of its query block.  When all splits of
+// a CTA parks its partial in shared memory — its own normalised result O / l in bf16 plus the
+// fp32 pair (m, l); the exchange of partials is bound by L2 bandwidth, so they travel in the
+// output's precision — sends it to the workspace with bulk copies (it stays in L2), and arrives
+// on a counter of its query block.  When all splits of
 // the block have arrived, every CTA fetches a slice of the rows of all partials with bulk copies
-// (plain loads would be throttled by the little L1 this kernel leaves), merges them, normalises
-// and writes bf16 output rows.  The launch is cooperative, so all CTAs are resident together and
+// (plain loads would be throttled by the little L1 this kernel leaves), combines them in fp32 with
+// the weights exp2(m_s - m) l_s / sum and writes bf16 output rows.  The launch is cooperative, so all CTAs are resident together and
 // the wait on the counter always ends; it is bounded all the same.  The counters live in the
 // tree object, start at zero and are put back to zero by the last CTA to leave.
 //
@@ -54,21 +56,19 @@ static_assert(2 * TC_REGS_SOFTMAX + TC_REGS_OTHER <= 3 * TC_REGS_LAUNCH, "setmax
 static_assert(TC_REGS_LAUNCH * TC_THREADS <= 65536, "launch register count does not fit the register file");
 
 // After the last key tile the Q / K / V buffers are reused:
-//   [0, 128 KB)      the parked partial O: 256 rows of 512 bytes; 16-byte chunk j of row r sits at
-//                    chunk position j ^ (r & 31), which makes the one-row-per-thread stores
-//                    conflict-free while rows stay contiguous for one bulk copy.  The workspace
-//                    holds partials in the same form; whoever reads a row undoes the permutation.
-//                    After the partial has left for the workspace the same space receives the
-//                    rows this CTA merges, from all splits.
-//   the last 8 KB    parked (m, l) per row; (m, l) then weights of every split for the merged
-//                    rows; 1 / l of the merged rows
-constexpr uint32_t TC_ROW_BYTES = 512;
+//   [0, 64 KB)       the parked partial: 256 rows of 128 bf16 values O / l (the split's own normalised
+//                    result; fp32 (m, l) travel beside it).  16-byte chunk j of row r sits at chunk
+//                    position j ^ (r & 15): the one-row-per-thread stores are conflict-free while rows
+//                    stay contiguous for one bulk copy.  The workspace holds partials in the same
+//                    form; whoever reads a row undoes the permutation.  After the partial has left
+//                    for the workspace the same space receives the rows this CTA merges.
+//   the last 8 KB    parked (m, l) per row; (m, l) then the merge weights of every split
+constexpr uint32_t TC_ROW_BYTES = 256;
 constexpr uint32_t TC_TILES_BYTES = TC_Q_BYTES + TC_RING_BYTES;
 constexpr uint32_t TC_PARK_ML_OFF = TC_TILES_BYTES - 8192;
 constexpr uint32_t TC_WBUF_OFF = TC_PARK_ML_OFF + 256 * 8;
 constexpr uint32_t TC_WBUF_ENTRIES = 256 + TC_MAX_SPLITS;
-constexpr uint32_t TC_ROWINV_OFF = TC_WBUF_OFF + TC_WBUF_ENTRIES * 8;
-static_assert(TC_ROWINV_OFF + 256 * 4 <= TC_TILES_BYTES, "merge buffers must fit the tile buffers");
+static_assert(TC_WBUF_OFF + TC_WBUF_ENTRIES * 8 <= TC_TILES_BYTES, "merge buffers must fit the tile buffers");
 static_assert((256 + TC_MAX_SPLITS) * TC_ROW_BYTES <= TC_PARK_ML_OFF, "rows to merge must fit below the small buffers");
 
 // barrier slots (8 bytes each) inside the barrier region
@@ -85,7 +85,7 @@ struct TcParams {
     const int32_t *seq_lens;
     const uint64_t *anc;   // [T][2]
     __nv_bfloat16 *out;    // [B][T][Hq][128]
-    float *ws_o;           // [groups][nsplit][256 rows][128] partial O, chunks permuted (only when nsplit > 1)
+    __nv_bfloat16 *ws_o;   // [groups][nsplit][256 rows][128] partial O / l, chunks permuted (only when nsplit > 1)
     float2 *ws_ml;         // [groups][nsplit][256] partial (m, l)
     int32_t *arrive, *depart;   // [groups] merge counters, zero between calls
     int32_t *status;       // [B] or null
@@ -160,9 +160,7 @@ struct TcCtx {
 template <bool SOFTMAX>
 __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    float2 *park_ml = reinterpret_cast<float2 *>(c.tiles + TC_PARK_ML_OFF);
     float2 *wbuf = reinterpret_cast<float2 *>(c.tiles + TC_WBUF_OFF);
-    float *rowinv = reinterpret_cast<float *>(c.tiles + TC_ROWINV_OFF);
     auto bar = [&](int i) { return c.bars + (uint32_t)i * 8u; };
 
     ptx::tc_fence_before();
@@ -191,22 +189,19 @@ __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
     const int nsplit = p.nsplit;
     const int grp = blockIdx.z * gridDim.y + blockIdx.y;
     const unsigned char *rows_smem = c.tiles;   // parked rows, later the rows to merge
-    // chunk j (16 bytes) of a 512-byte row whose index inside its 256-row slab is r
+    // chunk j (8 bf16 values) of a 256-byte row whose index inside its 256-row slab is r
     auto chunk = [&](const unsigned char *row_ptr, int r, int j) {
-        return *reinterpret_cast<const float4 *>(row_ptr + ((j ^ (r & 31)) << 4));
+        return *reinterpret_cast<const uint4 *>(row_ptr + ((j ^ (r & 15)) << 4));
+    };
+    auto out_ptr = [&](int r, int j) {   // 8 output values of query-block row r
+        const int node = r / p.G, hq = c.g * p.G + r % p.G;
+        return reinterpret_cast<uint4 *>(p.out + (((size_t)c.b * p.T + node) * p.Hq + hq) * 128 + j * 8);
     };
     if (nsplit == 1) {
-        // the partial is the result: normalise and store
-        for (int item = threadIdx.x; item < act_rows * 32; item += TC_THREADS) {
-            const int row = item / 32, c4 = item % 32, r = c.rows0 + row;
-            if (r >= p.M_rows) continue;
-            const float4 v = chunk(rows_smem + row * TC_ROW_BYTES, row, c4);
-            const float inv = 1.f / park_ml[row].y;
-            uint2 packed;
-            packed.x = pack2_bf16(v.x * inv, v.y * inv);
-            packed.y = pack2_bf16(v.z * inv, v.w * inv);
-            const int node = r / p.G, hq = c.g * p.G + r % p.G;
-            *reinterpret_cast<uint2 *>(p.out + (((size_t)c.b * p.T + node) * p.Hq + hq) * 128 + c4 * 4) = packed;
+        // the parked partial is the result
+        for (int item = threadIdx.x; item < act_rows * 16; item += TC_THREADS) {
+            const int row = item / 16, j = item % 16, r = c.rows0 + row;
+            if (r < p.M_rows) *out_ptr(r, j) = chunk(rows_smem + row * TC_ROW_BYTES, row, j);
         }
     } else {
         const size_t slab0 = (size_t)grp * nsplit;   // first slab of this query block
@@ -220,60 +215,67 @@ __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
             ptx::bulk_s2g(p.ws_ml + slab * 256, ptx::smem_u32(c.tiles + TC_PARK_ML_OFF), act_rows * 8);
             ptx::bulk_commit();
             ptx::bulk_wait_all();
+            TRACE(51);   // partial left shared memory and is written
             ptx::fence_proxy_async_all();
             __threadfence();
             atomicAdd(p.arrive + grp, 1);
+            TRACE(52);   // arrived
             const long long t0 = clock64();
             while (ld_acquire(p.arrive + grp) < nsplit)
                 if (clock64() - t0 > ptx::WAIT_CYCLE_LIMIT) { atomicExch(p.dev_error, MTV_ERR_TIMEOUT); break; }
+            TRACE(53);   // everybody arrived
             ptx::fence_proxy_async_all();
-            // ---- fetch rows [row_begin, row_begin + n_my) of every split: one bulk copy per split
-            if (n_my > 0) {
-                ptx::mbar_arrive_expect_tx(bar(BAR_MERGE), (uint32_t)(nsplit * n_my) * TC_ROW_BYTES);
-                for (int sp = 0; sp < nsplit; ++sp)
-                    ptx::bulk_g2s(ptx::smem_u32(c.tiles) + (uint32_t)(sp * n_my) * TC_ROW_BYTES,
-                                  p.ws_o + ((slab0 + sp) * 256 + row_begin) * 128, (uint32_t)n_my * TC_ROW_BYTES, bar(BAR_MERGE));
-            }
         }
         cta_sync();
+        // ---- fetch rows [row_begin, row_begin + n_my) of every split: one bulk copy per split, one lane each
+        if (warp == 0 && n_my > 0) {
+            if (lane == 0) ptx::mbar_arrive_expect_tx(bar(BAR_MERGE), (uint32_t)(nsplit * n_my) * TC_ROW_BYTES);
+            __syncwarp();
+            ptx::fence_proxy_async_all();   // the other CTAs' partials, acquired above, before the async-proxy reads
+            if (lane < nsplit)
+                ptx::bulk_g2s(ptx::smem_u32(c.tiles) + (uint32_t)(lane * n_my) * TC_ROW_BYTES,
+                              p.ws_o + ((slab0 + lane) * 256 + row_begin) * 128, (uint32_t)n_my * TC_ROW_BYTES, bar(BAR_MERGE));
+        }
         if (warp == 0) TRACE(45);   // all splits arrived, rows on their way
-        for (int idx = threadIdx.x; idx < n_my * nsplit; idx += TC_THREADS) {
-            const int rl = idx / nsplit, sp = idx - rl * nsplit;
-            wbuf[idx] = __ldcg(p.ws_ml + (slab0 + sp) * 256 + row_begin + rl);
+        // ---- merge weights, one warp per row, lane s = split s: exp2(m_s - m) l_s / sum over the splits
+        //      (split s contributes its own normalised result O_s / l_s)
+        for (int rl = warp; rl < n_my; rl += TC_THREADS / 32) {
+            float2 ml = make_float2(-INFINITY, 0.f);
+            if (lane < nsplit) ml = __ldcg(p.ws_ml + (slab0 + lane) * 256 + row_begin + rl);
+            float m = ml.x;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+            const float w = ml.x == -INFINITY ? 0.f : ex2(ml.x - m) * ml.y;
+            float lsum = w;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
+            if (lane < nsplit) wbuf[rl * nsplit + lane].x = w / lsum;
         }
         cta_sync();
-        for (int rl = threadIdx.x; rl < n_my; rl += TC_THREADS) {
-            float m = -INFINITY;
-            for (int sp = 0; sp < nsplit; ++sp) m = fmaxf(m, wbuf[rl * nsplit + sp].x);
-            float lsum = 0.f;
-            for (int sp = 0; sp < nsplit; ++sp) {
-                const float2 ml = wbuf[rl * nsplit + sp];
-                const float w = ml.x == -INFINITY ? 0.f : ex2(ml.x - m);
-                lsum += w * ml.y;
-                wbuf[rl * nsplit + sp].x = w;
-            }
-            rowinv[rl] = 1.f / lsum;
-        }
-        cta_sync();
+        if (warp == 0) TRACE(49);   // weights ready
         if (n_my > 0 && !ptx::mbar_wait(bar(BAR_MERGE), 0) && threadIdx.x == 0) atomicExch(p.dev_error, MTV_ERR_TIMEOUT);
-        for (int item = threadIdx.x; item < n_my * 32; item += TC_THREADS) {
-            const int rl = item / 32, c4 = item % 32;
+        if (warp == 0) TRACE(50);   // rows landed
+        for (int item = threadIdx.x; item < n_my * 16; item += TC_THREADS) {
+            const int rl = item / 16, j = item % 16;
             const int r = c.rows0 + row_begin + rl;
             if (r >= p.M_rows) continue;
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            float acc[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
             const unsigned char *row_ptr = rows_smem + rl * TC_ROW_BYTES;
+#pragma unroll 6
             for (int sp = 0; sp < nsplit; ++sp) {
                 const float w = wbuf[rl * nsplit + sp].x;
-                const float4 v = chunk(row_ptr + (size_t)(sp * n_my) * TC_ROW_BYTES, row_begin + rl, c4);
-                acc.x = fmaf(w, v.x, acc.x); acc.y = fmaf(w, v.y, acc.y);
-                acc.z = fmaf(w, v.z, acc.z); acc.w = fmaf(w, v.w, acc.w);
+                const uint4 v = chunk(row_ptr + (size_t)(sp * n_my) * TC_ROW_BYTES, row_begin + rl, j);
+                const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    acc[2 * e] = fmaf(w, __uint_as_float(vw[e] << 16), acc[2 * e]);
+                    acc[2 * e + 1] = fmaf(w, __uint_as_float(vw[e] & 0xffff0000u), acc[2 * e + 1]);
+                }
             }
-            const float inv = rowinv[rl];
-            uint2 packed;
-            packed.x = pack2_bf16(acc.x * inv, acc.y * inv);
-            packed.y = pack2_bf16(acc.z * inv, acc.w * inv);
-            const int node = r / p.G, hq = c.g * p.G + r % p.G;
-            *reinterpret_cast<uint2 *>(p.out + (((size_t)c.b * p.T + node) * p.Hq + hq) * 128 + c4 * 4) = packed;
+            *out_ptr(r, j) = make_uint4(pack2_bf16(acc[0], acc[1]), pack2_bf16(acc[2], acc[3]),
+                                        pack2_bf16(acc[4], acc[5]), pack2_bf16(acc[6], acc[7]));
         }
         if (warp == 0) TRACE(46);   // merge done
         // the last CTA of the query block to get here puts the counters back to zero
@@ -583,9 +585,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
             }
             const bool have_o = cnt > 0 && ok && !*abort_flag;
             {
-                // park the row: chunk j at position j ^ (row & 31); an empty split parks zeros
+                // park O / l of the row as bf16: chunk j at position j ^ (row & 15); an empty split parks zeros
                 unsigned char *dst = tiles_gen + (t * 128 + row) * TC_ROW_BYTES;
-                const int sw = (t * 128 + row) & 31;
+                const int sw = (t * 128 + row) & 15;
+                const float inv_l = have_o && l > 0.f ? 1.f / l : 0.f;
 #pragma unroll 1
                 for (int c = 0; c < 4; ++c) {
                     uint32_t o[32];
@@ -597,8 +600,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
                         for (int e = 0; e < 32; ++e) o[e] = 0u;
                     }
 #pragma unroll
-                    for (int e = 0; e < 32; e += 4)
-                        *reinterpret_cast<uint4 *>(dst + (((c * 8 + e / 4) ^ sw) << 4)) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
+                    for (int e = 0; e < 32; e += 8) {
+                        uint4 pk;
+                        pk.x = pack2_bf16(__uint_as_float(o[e]) * inv_l, __uint_as_float(o[e + 1]) * inv_l);
+                        pk.y = pack2_bf16(__uint_as_float(o[e + 2]) * inv_l, __uint_as_float(o[e + 3]) * inv_l);
+                        pk.z = pack2_bf16(__uint_as_float(o[e + 4]) * inv_l, __uint_as_float(o[e + 5]) * inv_l);
+                        pk.w = pack2_bf16(__uint_as_float(o[e + 6]) * inv_l, __uint_as_float(o[e + 7]) * inv_l);
+                        *reinterpret_cast<uint4 *>(dst + (((c * 4 + e / 8) ^ sw) << 4)) = pk;
+                    }
                 }
                 park_ml[t * 128 + row] = make_float2(m_used, l);   // (-inf, 0) for an empty split
                 ptx::fence_proxy_async();   // the bulk copy out of shared memory must see these stores
@@ -675,7 +684,7 @@ int attn_tc_plan(int T, int G, int B, int Hkv, int Lcap, int *n_rt_out) {
 
 int launch_tree_attn_tc(const mtv_tree *tree, int B, int Hq, int Hkv, const __nv_bfloat16 *q, const __nv_bfloat16 *k,
                         const __nv_bfloat16 *v, int64_t sb, int64_t sh, int64_t st, int Lcap, const int32_t *seq_lens,
-                        float scale_log2, __nv_bfloat16 *out, int32_t *status, float *ws_o, float *ws_ml,
+                        float scale_log2, __nv_bfloat16 *out, int32_t *status, void *ws_o, float *ws_ml,
                         cudaStream_t stream) {
     const int G = Hq / Hkv, T = tree->T, D = 128;
     CUtensorMap q_map, k_map, v_map;
@@ -694,7 +703,7 @@ int launch_tree_attn_tc(const mtv_tree *tree, int B, int Hq, int Hkv, const __nv
     if (tc_prepare() != MTV_OK) return MTV_ERR_CUDA;
     TcParams p;
     p.seq_lens = seq_lens; p.anc = tree->d_anc; p.out = out; p.status = status; p.dev_error = tree->d_error;
-    p.ws_o = ws_o; p.ws_ml = reinterpret_cast<float2 *>(ws_ml);
+    p.ws_o = reinterpret_cast<__nv_bfloat16 *>(ws_o); p.ws_ml = reinterpret_cast<float2 *>(ws_ml);
     p.arrive = tree->d_counters; p.depart = tree->d_counters + TC_MAX_GROUPS;
     p.scale_log2 = scale_log2;
     p.T = T; p.G = G; p.Hq = Hq; p.Hkv = Hkv; p.Lcap = Lcap;
