@@ -38,6 +38,8 @@ def parse():
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-taps", action="store_true", help="skip per-kernel event timing")
+    ap.add_argument("--launch", default="graph", choices=["graph", "stream"],
+                    help="timed steps: replay of one captured CUDA graph per step, or plain stream launches")
     return ap.parse_args()
 
 
@@ -99,7 +101,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.QUERY,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -224,21 +226,40 @@ def run_ours(args):
     for _ in range(W_steps):
         step()
     barrier()
+    # per-kernel durations: an untimed pass of stream launches with the library's event taps
+    taps = None
+    tap_steps = min(K_steps, 10)
+    if not args.no_taps:
+        taps = binding.KernelTaps(tap_steps * n_layers)
+        taps.__enter__()
+        for _ in range(tap_steps):
+            step()
+        barrier()
+        taps.__exit__()
+    # the timed steps
+    run_step = step
+    if args.launch == "graph":
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                step()
+        torch.cuda.current_stream().wait_stream(side)
+        run_step = graph.replay
+        for _ in range(2):
+            run_step()
+        barrier()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    taps = None if args.no_taps else binding.KernelTaps(K_steps * n_layers)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if taps:
-        taps.__enter__()
     barrier()
     e0.record()
     for _ in range(K_steps):
-        step()
+        run_step()
     e1.record()
     barrier()
-    if taps:
-        taps.__exit__()
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None
     ms_total = max_over_ranks(ms_total, world, dev)
@@ -282,7 +303,8 @@ def run_ours(args):
             w.name, w.B, w.L_lo if w.L_lo == w.L_hi else "U[%d,%d]" % (w.L_lo, w.L_hi), w.H, w.Hq, w.Hkv, w.D, w.V,
             w.K, tree.T, n_layers),
             "l2": "inputs larger than L2: %.2f GB streamed per step, %d distinct KV caches" % (alg["step"] / 1e9, n_layers),
-            "launch": "stream launches through mtv_verify_step", "seed": w.seed,
+            "launch": ("one CUDA graph per step (captured mtv_verify_step), replayed" if args.launch == "graph"
+                       else "stream launches through mtv_verify_step"), "seed": w.seed,
             "mean_tokens_per_step": mean_tokens, "context": PAPER_CONTEXT},
         "clocks": clocks,
         "e2e": {"value": world / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -295,7 +317,7 @@ def run_ours(args):
     if taps:
         tm = taps.times_ms()
         avg = {k: (sum(v) / len(v) if v else None) for k, v in tm.items()}
-        per_step = {k: (sum(v) / K_steps if v else 0.0) for k, v in tm.items()}
+        per_step = {k: (sum(v) / tap_steps if v else 0.0) for k, v in tm.items()}
         out["kernel_ms_per_step"] = per_step
         dom = max(per_step, key=per_step.get)
         bytes_of = {"heads_vocab_topk": alg["heads_vocab"], "attn_partial": alg["attn_per_layer"],
@@ -305,7 +327,7 @@ def run_ours(args):
                            "frac": ach / pk["hbm_gbs"], "traffic": measured_traffic(dom), "peak_source": pk["source"],
                            "algorithmic_bytes_per_launch": bytes_of.get(dom, 0), "avg_launch_ms": avg[dom]}
         a_ms = (avg["attn_partial"] or 0.0) + (avg["attn_combine"] or 0.0)
-        out["gpu_launches"] = sum(len(v) for v in tm.values())
+        out["gpu_launches"] = sum(len(v) for v in tm.values()) * K_steps // tap_steps
         ach = alg["attn_per_layer"] / a_ms / 1e6
         out["roofline_attn"] = {"kernel": "tree_verify_attention (all its launches)", "bound": "hbm", "achieved": ach,
                                 "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": ach / pk["hbm_gbs"],
