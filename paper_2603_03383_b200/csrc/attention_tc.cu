@@ -21,7 +21,7 @@
 // on a counter of its query block.  When all splits of
 // the block have arrived, every CTA fetches a slice of the rows of all partials with bulk copies
 // (plain loads would be throttled by the little L1 this kernel leaves), combines them in fp32 with
-// the weights exp2(m_s - m) l_s / sum and writes bf16 output rows.  The launch is cooperative, so all CTAs are resident together and
+// the weights exp2(m_s - m) l_s / sum and writes bf16 output rows.  The grid never exceeds one CTA per SM, so all CTAs are resident together and
 // the wait on the counter always ends; it is bounded all the same.  The counters live in the
 // tree object, start at zero and are put back to zero by the last CTA to leave.
 //
@@ -296,6 +296,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                     const __grid_constant__ CUtensorMap v_map, const TcParams p) {
     extern __shared__ unsigned char smem_raw[];
+    // Programmatic dependent launch: let the next kernel of the stream be set up while this one runs,
+    // and do not touch global memory before the previous kernel has completed.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int split = blockIdx.x;
     const int g = blockIdx.y / p.n_rt, rt = blockIdx.y % p.n_rt;
     const int b = blockIdx.z;
@@ -714,9 +718,15 @@ int launch_tree_attn_tc(const mtv_tree *tree, int B, int Hq, int Hkv, const __nv
     cfg.blockDim = dim3(TC_THREADS, 1, 1);
     cfg.dynamicSmemBytes = TC_SMEM_BYTES;
     cfg.stream = stream;
+    // Launched as a programmatic dependent of the previous kernel in the stream (the kernel itself
+    // waits for that kernel before it reads anything), which hides most of the launch latency when
+    // attention calls follow each other.  Not a cooperative launch: that costs about 2 us per
+    // launch; the grid never exceeds one CTA per SM, so its CTAs are resident together whenever the
+    // device is not shared with another long-running kernel, and the wait for the other splits is
+    // bounded in any case.
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;   // CTAs that wait for each other must all be resident
-    attr[0].val.cooperative = p.nsplit > 1 ? 1 : 0;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     MTV_CUDA_CHECK(cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel, q_map, k_map, v_map, p));
     return MTV_OK;
