@@ -2,17 +2,18 @@
 //
 // One CTA owns up to 256 query rows (two 128-row tiles of the (node, head-in-group) block
 // that shares one KV head) and a contiguous range of 128-key tiles.  Warp roles:
-//   warps 0-3 / 4-7  softmax warpgroup of row tile 0 / 1: one thread per query row reads its
-//                    row of S from tensor memory, applies the ancestor bitmask on the tiles that
-//                    overlap the tree rows, keeps a running (max, sum) and writes P (bf16) back
-//                    to tensor memory over S;
-//   warp 8           issues tcgen05.mma: S_t = Q_t K^T (operands in shared memory) and
+//   warps 0-7 / 8-15 softmax warps of row tile 0 / 1: two threads per query row, each with one
+//                    half (64 keys) of the row of S from tensor memory in registers — two such warps
+//                    per scheduler, so that one can use the special-function unit while the other
+//                    issues the rest; they apply the ancestor bitmask on the tiles that overlap the
+//                    tree rows, agree on the running max through shared memory, keep partial row
+//                    sums and write P (bf16) back to tensor memory over S;
+//   warp 16          issues tcgen05.mma: S_t = Q_t K^T (operands in shared memory) and
 //                    O_t += P_t V (P from tensor memory, V from shared memory, N-major);
-//   warp 9           TMA producer: Q once, then K and V tiles through a ring of 32 KB slots;
-//   warps 10-11      only help with the copies of the merge.
+//   warp 17          TMA producer: Q once, then K and V tiles through a ring of 32 KB slots;
+//   warps 18-19      only help with the copies of the merge.
 // Tensor memory: S0 | S1 | O0 | O1, 128 fp32 columns each; P_t overlays the first 64 columns
-// of S_t.  The softmax warpgroups take registers from the third warpgroup (setmaxnreg), so a
-// thread holds its whole row of S.
+// of S_t.  The softmax warpgroups take registers from the fifth warpgroup (setmaxnreg).
 //
 // The key splits of one query block are merged inside the same launch.  After its last key tile
 // a CTA parks its partial in shared memory — its own normalised result O / l in bf16 plus the
@@ -36,23 +37,26 @@ namespace mtv {
 
 constexpr int TC_BN = 128;
 constexpr int TC_SLOTS = 5;
-constexpr int TC_THREADS = 384;   // 3 warpgroups: softmax 0, softmax 1, {MMA warp, TMA warp, 2 helper warps}
+constexpr int TC_THREADS = 640;   // 5 warpgroups: 4 of softmax warps, {MMA warp, TMA warp, 2 helper warps}
+constexpr int TC_MMA_WARP = 16, TC_TMA_WARP = 17;
 constexpr uint32_t TC_TILE_BYTES = 128 * 128 * 2;   // one 128 x 128 bf16 tile: two 64-column halves
 constexpr uint32_t TC_HALF_BYTES = TC_TILE_BYTES / 2;
 constexpr uint32_t TC_Q_BYTES = 2 * TC_TILE_BYTES;
 constexpr uint32_t TC_RING_BYTES = TC_SLOTS * TC_TILE_BYTES;
 constexpr uint32_t TC_BAR_BYTES = 256;
-constexpr uint32_t TC_SMEM_BYTES = 1024 + TC_Q_BYTES + TC_RING_BYTES + TC_BAR_BYTES;
+constexpr uint32_t TC_XMAX_BYTES = 2 * 2 * 128 * 2;   // running-max exchange of the two half-row threads, bf16
+constexpr uint32_t TC_SMEM_BYTES = 1024 + TC_Q_BYTES + TC_RING_BYTES + TC_BAR_BYTES + TC_XMAX_BYTES;
+static_assert(TC_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 constexpr float TC_RESCALE_THRESHOLD = 8.f;
 constexpr int TC_MAX_SPLITS = 32;
 constexpr int TC_MAX_GROUPS = 256;   // merge counters available in the tree object
 
 // Register rebalancing.  The CTA's pool is what the launch allocates: TC_THREADS threads at the
-// per-thread count the compiler derives from the launch bounds (65536 / 384 rounded down to a
-// multiple of 8 = 168).  setmaxnreg.inc blocks until the pool has the registers, so the three
-// warpgroups' targets must not add up to more than the pool: 2 x 216 + 72 = 3 x 168.
-constexpr int TC_REGS_LAUNCH = 168, TC_REGS_SOFTMAX = 216, TC_REGS_OTHER = 72;
-static_assert(2 * TC_REGS_SOFTMAX + TC_REGS_OTHER <= 3 * TC_REGS_LAUNCH, "setmaxnreg targets exceed the CTA's register pool");
+// per-thread count the compiler derives from the launch bounds (65536 / 640 rounded down to a
+// multiple of 8 = 96).  setmaxnreg.inc blocks until the pool has the registers, so the five
+// warpgroups' targets must not add up to more than the pool: 4 x 104 + 64 = 5 x 96.
+constexpr int TC_REGS_LAUNCH = 96, TC_REGS_SOFTMAX = 104, TC_REGS_OTHER = 64;
+static_assert(4 * TC_REGS_SOFTMAX + TC_REGS_OTHER <= 5 * TC_REGS_LAUNCH, "setmaxnreg targets exceed the CTA's register pool");
 static_assert(TC_REGS_LAUNCH * TC_THREADS <= 65536, "launch register count does not fit the register file");
 
 // After the last key tile the Q / K / V buffers are reused:
@@ -171,11 +175,11 @@ __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
         // the other splits never wait for it; the error word tells the host the output is invalid.
         if (threadIdx.x == 0) atomicExch(p.dev_error, MTV_ERR_TIMEOUT);
         if (!SOFTMAX) {
-            if (warp == 9 && lane == 0) {
+            if (warp == TC_TMA_WARP && lane == 0) {
                 ptx::mbar_wait(bar(BAR_Q), 0);
                 for (int s = 0; s < TC_SLOTS; ++s) { ptx::mbar_wait(bar(BAR_KV_FULL + s), 0); ptx::mbar_wait(bar(BAR_KV_FULL + s), 1); }
             }
-            if (warp == 8) {
+            if (warp == TC_MMA_WARP) {
                 if (!c.final_committed && lane == 0) ptx::tc_commit(bar(BAR_FINAL));
                 __syncwarp();
                 ptx::mbar_wait(bar(BAR_FINAL), 0);
@@ -285,7 +289,7 @@ __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
             __threadfence();
         }
     }
-    if (!SOFTMAX && warp == 8) {
+    if (!SOFTMAX && warp == TC_MMA_WARP) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(c.tmem, 512);
     }
@@ -345,12 +349,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     const int n_loads = 2 * cnt;
     const int n_early = min(n_loads, TC_SLOTS);   // loads that need no free slot: issued before the CTA syncs
 
-    if (warp == 9 && lane == 0) {
+    if (warp == TC_TMA_WARP && lane == 0) {
         ptx::mbar_init(bar(BAR_Q), 1);
         for (int s = 0; s < TC_SLOTS; ++s) { ptx::mbar_init(bar(BAR_KV_FULL + s), 1); ptx::mbar_init(bar(BAR_KV_EMPTY + s), 1); }
         for (int t = 0; t < 2; ++t) {
             ptx::mbar_init(bar(BAR_S + t), 1);
-            ptx::mbar_init(bar(BAR_P + t), 128);
+            ptx::mbar_init(bar(BAR_P + t), 256);
             ptx::mbar_init(bar(BAR_O + t), 1);
         }
         ptx::mbar_init(bar(BAR_FINAL), 1);
@@ -368,7 +372,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
             for (int i = 1; i < n_early; ++i) issue_kv(i);
         }
     }
-    if (warp == 8) {
+    if (warp == TC_MMA_WARP) {
         ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t *>(tmem_slot)), 512);
         ptx::tmem_relinquish();
     }
@@ -383,9 +387,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     ctx.final_committed = false;
     const uint32_t tmem = ctx.tmem;
 
-    if (warp >= 8) {
-        reg_dec<TC_REGS_OTHER>();   // the whole third warpgroup gives registers to the softmax warpgroups
-        if (warp == 9) {
+    if (warp >= 16) {
+        reg_dec<TC_REGS_OTHER>();   // the whole fifth warpgroup gives registers to the softmax warpgroups
+        if (warp == TC_TMA_WARP) {
             // ------------------------------------------------------------ TMA producer (the rest of the tiles)
             for (int i = n_early; i < n_loads && !*abort_flag; ++i) {
                 const int slot = i % TC_SLOTS, use = i / TC_SLOTS;
@@ -393,7 +397,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
                 if (lane == 0) issue_kv(i);
                 __syncwarp();
             }
-        } else if (warp == 8) {
+        } else if (warp == TC_MMA_WARP) {
             // ------------------------------------------------------------ MMA issuer
             auto issue_S = [&](int t, int j) {
                 const uint32_t kbase = ring + ((2 * j) % TC_SLOTS) * TC_TILE_BYTES;
@@ -481,15 +485,20 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
         tc_epilogue<false>(p, ctx);
     } else {
         reg_inc<TC_REGS_SOFTMAX>();
-        if (warp / 4 < nt) {
-            // ------------------------------------------------------------ softmax warpgroup of row tile t
-            const int t = warp / 4;
+        if (warp / 8 < nt) {
+            // ------------------------------------------------------------ softmax warps of row tile t
+            // Thread (row, hf) owns keys [64 hf, 64 hf + 64) of its query row in every key tile.
+            const int t = warp / 8, hf = (warp / 4) & 1;
             const int row = (warp % 4) * 32 + lane;
             const int r = rows0 + t * 128 + row;
             uint64_t alo = 0, ahi = 0;
             if (r < p.M_rows) { alo = p.anc[(r / p.G) * 2]; ahi = p.anc[(r / p.G) * 2 + 1]; }
-            const uint32_t t_s = tmem + ((uint32_t)((warp % 4) * 32) << 16) + t * 128;
-            const uint32_t t_o = tmem + ((uint32_t)((warp % 4) * 32) << 16) + 256 + t * 128;
+            const uint32_t lane_base = (uint32_t)((warp % 4) * 32) << 16;
+            const uint32_t t_s = tmem + lane_base + t * 128 + hf * 64;          // this thread's 64 columns of S_t
+            const uint32_t t_p = tmem + lane_base + t * 128 + hf * 32;          // its 32 columns of P_t
+            const uint32_t t_o = tmem + lane_base + 256 + t * 128 + hf * 64;    // its 64 columns of O_t
+            __nv_bfloat16 *xmax = reinterpret_cast<__nv_bfloat16 *>(bar_region + TC_BAR_BYTES);   // [t][hf][row]
+            auto pair_sync = [&]() { asm volatile("bar.sync %0, 256;" ::"r"(2 + t) : "memory"); };  // the 256 threads of row tile t
             float m_used = -INFINITY, l = 0.f;
             bool ok = true;
             // visibility of the tree rows as 32-bit words: word q covers tree rows 32q .. 32q+31
@@ -501,21 +510,23 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
                 if (q == 3) return (uint32_t)(ahi >> 32);
                 return 0u;                         // past the tree rows: nothing
             };
-            for (int j = 0; j < cnt && !*abort_flag; ++j) {
-                ok = ptx::mbar_wait(bar(BAR_S + t), j & 1);
-                if (!ok) break;
-                if (warp % 4 == 0 && j < 6) TRACE(8 + t * 16 + j * 2);       // S_t(j) ready
+            // A thread whose wait ran out keeps going through the motions without waiting, so that
+            // the barriers it shares with the other half-row threads stay matched.
+            for (int j = 0; j < cnt; ++j) {
+                if (*abort_flag) ok = false;
+                if (ok) ok = ptx::mbar_wait(bar(BAR_S + t), j & 1);
+                if (warp % 8 == 0 && j < 6) TRACE(8 + t * 16 + j * 2);       // S_t(j) ready
                 ptx::tc_fence_after();
-                // ---- the whole row of S in registers (raw scores; the scale is positive)
-                uint32_t sr[4][32];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) ptx::tmem_ld32(t_s + c * 32, sr[c]);
+                // ---- this thread's half row of S in registers (raw scores; the scale is positive)
+                uint32_t sr[2][32];
+                ptx::tmem_ld32(t_s, sr[0]);
+                ptx::tmem_ld32(t_s + 32, sr[1]);
                 ptx::tmem_ld_wait();
-                const int key0 = (t_begin + j) * TC_BN;
-                if (key0 + TC_BN > L) {
-                    // tile overlaps the tree rows or the end of the cache: bit e of vis is column 32c + e
+                const int key0 = (t_begin + j) * TC_BN + hf * 64;
+                if (key0 + 64 > L) {
+                    // the half tile overlaps the tree rows or the end of the cache: bit e of vis is column 32c + e
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
+                    for (int c = 0; c < 2; ++c) {
                         const int a0 = key0 + c * 32 - L;        // tree row of the chunk's first column
                         const int q = a0 >> 5, sh = a0 & 31;     // floor division
                         const uint32_t vis = __funnelshift_r(anc_word(q), anc_word(q + 1), sh);
@@ -526,7 +537,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
                 }
                 float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
+                for (int c = 0; c < 2; ++c)
 #pragma unroll
                     for (int e = 0; e < 32; e += 4) {
                         mx0 = fmaxf(mx0, __uint_as_float(sr[c][e]));
@@ -534,17 +545,21 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
                         mx2 = fmaxf(mx2, __uint_as_float(sr[c][e + 2]));
                         mx3 = fmaxf(mx3, __uint_as_float(sr[c][e + 3]));
                     }
-                const float mxs = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
+                // The two halves need the same reference, not the exact maximum (P may reach 2^8):
+                // they exchange their maxima rounded to bf16 and both take the larger rounded value.
+                const __nv_bfloat16 own = __float2bfloat16_rn(fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
+                xmax[(t * 2 + hf) * 128 + row] = own;
+                pair_sync();   // also: both halves hold their S before anyone overwrites it with P
+                const float mxs = fmaxf(__bfloat162float(own), __bfloat162float(xmax[(t * 2 + (hf ^ 1)) * 128 + row]));
                 const float m_new = (j == 0 || mxs > m_used + TC_RESCALE_THRESHOLD) ? mxs : m_used;
                 // O holds sums relative to m_used: rescale it when the reference moves (rare)
                 const bool need = j > 0 && m_new != m_used && m_used != -INFINITY;
                 if (__any_sync(0xffffffffu, need)) {
-                    ok = ptx::mbar_wait(bar(BAR_O + t), (j - 1) & 1);
-                    if (!ok) break;
+                    if (ok) ok = ptx::mbar_wait(bar(BAR_O + t), (j - 1) & 1);
                     ptx::tc_fence_after();
                     const float alpha = need ? ex2(m_used - m_new) : 1.f;
 #pragma unroll 1
-                    for (int c = 0; c < 8; ++c) {
+                    for (int c = 0; c < 4; ++c) {
                         uint32_t o[16];
                         ptx::tmem_ld16(t_o + c * 16, o);
                         ptx::tmem_ld_wait();
@@ -557,10 +572,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
                 }
                 m_used = m_new;
                 const float m_eff = m_used == -INFINITY ? 0.f : m_used;
-                // ---- P = exp2(scale * S - m), row sum, bf16 P over the first 64 columns of S
+                // ---- P = exp2(scale * S - m), partial row sum, bf16 P over the first 64 columns of S_t
                 float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < 2; ++c) {
                     uint32_t pk[16];
 #pragma unroll
                     for (int e = 0; e < 16; e += 2) {
@@ -572,29 +587,36 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
                         pk[e] = pack2_bf16(p0, p1);
                         pk[e + 1] = pack2_bf16(p2, p3);
                     }
-                    ptx::tmem_st16(t_s + c * 16, pk);
+                    ptx::tmem_st16(t_p + c * 16, pk);
                 }
                 l += (l0 + l1) + (l2 + l3);
                 ptx::tmem_st_wait();
                 ptx::tc_fence_before();
                 ptx::mbar_arrive(bar(BAR_P + t));
-                if (warp % 4 == 0 && j < 6) TRACE(9 + t * 16 + j * 2);       // P_t(j) written
+                if (warp % 8 == 0 && j < 6) TRACE(9 + t * 16 + j * 2);       // P_t(j) written
             }
             // ---- hand over the partial of this row
             if (cnt > 0) {
                 // every tensor-core read of the tile buffers must be over before they are reused
-                if (ok && !*abort_flag) ok = ptx::mbar_wait(bar(BAR_FINAL), 0);
-                if (warp % 4 == 0) TRACE(40 + t);                            // all tensor-core work done
-                if (ok) ptx::tc_fence_after();
+                if (*abort_flag) ok = false;
+                if (ok) ok = ptx::mbar_wait(bar(BAR_FINAL), 0);
+                if (warp % 8 == 0) TRACE(40 + t);                            // all tensor-core work done
+                ptx::tc_fence_after();
             }
-            const bool have_o = cnt > 0 && ok && !*abort_flag;
+            // the row sum is the sum of the two halves' sums
+            float *lx = reinterpret_cast<float *>(tiles_gen + TC_WBUF_OFF);   // [t][hf][row], free once the tiles are
+            lx[(t * 2 + hf) * 128 + row] = l;
+            pair_sync();
+            l += lx[(t * 2 + (hf ^ 1)) * 128 + row];
+            const bool have_o = cnt > 0 && ok;
             {
-                // park O / l of the row as bf16: chunk j at position j ^ (row & 15); an empty split parks zeros
+                // park this thread's 64 columns of O / l as bf16: chunk j at position j ^ (row & 15); an empty
+                // split parks zeros
                 unsigned char *dst = tiles_gen + (t * 128 + row) * TC_ROW_BYTES;
                 const int sw = (t * 128 + row) & 15;
                 const float inv_l = have_o && l > 0.f ? 1.f / l : 0.f;
 #pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < 2; ++c) {
                     uint32_t o[32];
                     if (have_o) {
                         ptx::tmem_ld32(t_o + c * 32, o);
@@ -610,10 +632,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
                         pk.y = pack2_bf16(__uint_as_float(o[e + 2]) * inv_l, __uint_as_float(o[e + 3]) * inv_l);
                         pk.z = pack2_bf16(__uint_as_float(o[e + 4]) * inv_l, __uint_as_float(o[e + 5]) * inv_l);
                         pk.w = pack2_bf16(__uint_as_float(o[e + 6]) * inv_l, __uint_as_float(o[e + 7]) * inv_l);
-                        *reinterpret_cast<uint4 *>(dst + (((c * 4 + e / 8) ^ sw) << 4)) = pk;
+                        *reinterpret_cast<uint4 *>(dst + (((hf * 8 + c * 4 + e / 8) ^ sw) << 4)) = pk;
                     }
                 }
-                park_ml[t * 128 + row] = make_float2(m_used, l);   // (-inf, 0) for an empty split
+                if (hf == 0) park_ml[t * 128 + row] = make_float2(m_used, l);   // (-inf, 0) for an empty split
                 ptx::fence_proxy_async();   // the bulk copy out of shared memory must see these stores
             }
             if (!ok) *abort_flag = 1;
