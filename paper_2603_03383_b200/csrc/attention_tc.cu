@@ -300,27 +300,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                     const __grid_constant__ CUtensorMap v_map, const TcParams p) {
     extern __shared__ unsigned char smem_raw[];
-    // Programmatic dependent launch: let the next kernel of the stream be set up while this one runs,
-    // and do not touch global memory before the previous kernel has completed.
+    // Programmatic dependent launch: let the next kernel of the stream be set up while this one runs.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int split = blockIdx.x;
     const int g = blockIdx.y / p.n_rt, rt = blockIdx.y % p.n_rt;
     const int b = blockIdx.z;
-    const int L = p.seq_lens[b];
-    const bool reporter = blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0;
-    if (L + p.T > p.Lcap) {         // the same for every CTA of the query block: nobody waits for anybody
-        if (reporter && p.status) p.status[b] = MTV_ERR_CAPACITY;
-        return;
-    }
-    if (reporter && p.status) p.status[b] = MTV_OK;
-    const int n_keys = L + p.T;
-    const int tiles = (n_keys + TC_BN - 1) / TC_BN;
-    const int base_cnt = tiles / p.nsplit, rem = tiles % p.nsplit;
-    const int t_begin = split * base_cnt + min(split, rem);
-    const int cnt = base_cnt + (split < rem ? 1 : 0);
-    const int rows0 = rt * 256;
-    const int nt = p.M_rows - rows0 > 128 ? 2 : 1;
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     if (warp == 0) TRACE(0);
 
@@ -337,6 +321,47 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     auto bar = [&](int i) { return bars + (uint32_t)i * 8u; };
     float2 *park_ml = reinterpret_cast<float2 *>(tiles_gen + TC_PARK_ML_OFF);
 
+    if (warp == TC_TMA_WARP && lane == 0) {
+        ptx::mbar_init(bar(BAR_Q), 1);
+        for (int s = 0; s < TC_SLOTS; ++s) { ptx::mbar_init(bar(BAR_KV_FULL + s), 1); ptx::mbar_init(bar(BAR_KV_EMPTY + s), 1); }
+        for (int t = 0; t < 2; ++t) {
+            ptx::mbar_init(bar(BAR_S + t), 1);
+            ptx::mbar_init(bar(BAR_P + t), 256);
+            ptx::mbar_init(bar(BAR_O + t), 1);
+        }
+        ptx::mbar_init(bar(BAR_FINAL), 1);
+        ptx::mbar_init(bar(BAR_MERGE), 1);
+        ptx::fence_mbar_init();
+        *abort_flag = 0;
+    }
+    if (warp == TC_MMA_WARP) {
+        ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t *>(tmem_slot)), 512);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    if (warp == 0) TRACE(1);
+
+    // Nothing above touched global memory.  From here on the previous kernel of the stream must be
+    // complete (its outputs may be this kernel's inputs, and it may share the workspace and counters).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int L = p.seq_lens[b];
+    const bool reporter = blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0;
+    if (L + p.T > p.Lcap) {         // the same for every CTA of the query block: nobody waits for anybody
+        if (reporter && p.status) p.status[b] = MTV_ERR_CAPACITY;
+        if (warp == TC_MMA_WARP) ptx::tmem_dealloc(*tmem_slot, 512);
+        return;
+    }
+    if (reporter && p.status) p.status[b] = MTV_OK;
+    const int n_keys = L + p.T;
+    const int tiles = (n_keys + TC_BN - 1) / TC_BN;
+    const int base_cnt = tiles / p.nsplit, rem = tiles % p.nsplit;
+    const int t_begin = split * base_cnt + min(split, rem);
+    const int cnt = base_cnt + (split < rem ? 1 : 0);
+    const int rows0 = rt * 256;
+    const int nt = p.M_rows - rows0 > 128 ? 2 : 1;
+
     // One K or V tile into ring slot (i mod TC_SLOTS): i = 2j is K of key tile j, i = 2j + 1 is V.
     auto issue_kv = [&](int i) {
         const int slot = i % TC_SLOTS;
@@ -350,17 +375,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     const int n_early = min(n_loads, TC_SLOTS);   // loads that need no free slot: issued before the CTA syncs
 
     if (warp == TC_TMA_WARP && lane == 0) {
-        ptx::mbar_init(bar(BAR_Q), 1);
-        for (int s = 0; s < TC_SLOTS; ++s) { ptx::mbar_init(bar(BAR_KV_FULL + s), 1); ptx::mbar_init(bar(BAR_KV_EMPTY + s), 1); }
-        for (int t = 0; t < 2; ++t) {
-            ptx::mbar_init(bar(BAR_S + t), 1);
-            ptx::mbar_init(bar(BAR_P + t), 256);
-            ptx::mbar_init(bar(BAR_O + t), 1);
-        }
-        ptx::mbar_init(bar(BAR_FINAL), 1);
-        ptx::mbar_init(bar(BAR_MERGE), 1);
-        ptx::fence_mbar_init();
-        *abort_flag = 0;
         if (cnt > 0) {
             // first K tile, then Q, then the rest: the first MMA needs K_0 and Q
             issue_kv(0);
@@ -372,14 +386,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
             for (int i = 1; i < n_early; ++i) issue_kv(i);
         }
     }
-    if (warp == TC_MMA_WARP) {
-        ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t *>(tmem_slot)), 512);
-        ptx::tmem_relinquish();
-    }
-    ptx::tc_fence_before();
-    __syncthreads();
-    ptx::tc_fence_after();
-    if (warp == 0) TRACE(1);
+    __syncwarp();
 
     TcCtx ctx;
     ctx.tiles = tiles_gen; ctx.bars = bars; ctx.abort_flag = abort_flag; ctx.tmem = *tmem_slot;

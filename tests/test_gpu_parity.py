@@ -111,9 +111,10 @@ def test_attention_ragged_batch_many_splits_and_strided_cache():
     _attention_case(tb, tree, 3, 8, 2, 128, [1500, 40, 777], seed=9, Lcap=1600, pad=24)
 
 
-def test_attention_capacity_is_reported_not_faulted():
+@pytest.mark.parametrize("D", [64, 128])
+def test_attention_capacity_is_reported_not_faulted(D):
     tb, tree = make_tree("cartesian", 2, (2, 2))
-    T, B, Hq, Hkv, D, Lcap = tree.T, 2, 4, 2, 64, 40
+    T, B, Hq, Hkv, Lcap = tree.T, 2, 4, 2, 40
     q, k, v = synth.attention_inputs(B, T, Hq, Hkv, D, Lcap, 3, device=DEV)
     sl = torch.tensor([Lcap - T + 1, 10], dtype=torch.int32, device=DEV)       # first sequence does not fit
     out = torch.full((B, T, Hq, D), 3.0, dtype=torch.bfloat16, device=DEV)
@@ -125,6 +126,12 @@ def test_attention_capacity_is_reported_not_faulted():
     assert bool((out[0] == 3.0).all())                                          # untouched
     want = ref.tree_attention(q[1:].cpu(), k[1:].cpu(), v[1:].cpu(), sl[1:].cpu(), tb["mask"])
     assert_close(out[1:], want)
+    # and the next call on the same device works (nothing was left allocated or half-synchronised)
+    sl2 = torch.tensor([5, 10], dtype=torch.int32, device=DEV)
+    binding.tree_verify_attention(tree, q, k, v, sl2, out, ws, status=status)
+    torch.cuda.synchronize()
+    assert status.tolist() == [0, 0] and binding.mtv_device_error(tree) == 0
+    assert_close(out, ref.tree_attention(q.cpu(), k.cpu(), v.cpu(), sl2.cpu(), tb["mask"]))
 
 
 @pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 128), (8, 2, 64)])
@@ -321,3 +328,61 @@ def test_generator_is_identical_on_cpu_and_gpu():
     b = synth.normal_bf16(123, 5, (1 << 16,), 0.37, device=DEV)
     assert torch.equal(a, b.cpu())
     assert torch.equal(synth.uniform_int(9, 1, 100, 5, 5000), synth.uniform_int(9, 1, 100, 5, 5000, device=DEV).cpu())
+
+
+def test_full_step_replays_from_a_cuda_graph():
+    """The whole step only enqueues work (no host synchronisation, no allocation): it can be captured once
+    and replayed, and the replay gives what the oracle gives."""
+    w = synth.WORKLOADS["tiny"]
+    tb, tree = make_tree(w.tree, w.K, w.topk, w.T)
+    T, B, K, n_layers = tree.T, 2, w.K, 2
+    lens = [100, 37]
+    Lcap = max(lens) + T
+    seed, inp, cpu, cand_ref, cl_ref, tt_ref = oracle_heads_with_margin(B, 256, 2000, K, tb, 41)
+    logits, planted = synth.planted_logits(B, T, 2000, K, tt_ref, tb["parent"], tb["rank"], seed, p_accept=(0.9,))
+    acc_ref = ref.tree_accept(ref.node_argmax(logits), tt_ref, tb)
+    sl = torch.tensor(lens, dtype=torch.int32)
+    layers = [synth.attention_inputs(B, T, 8, 2, 128, Lcap, seed, layer=l) for l in range(n_layers)]
+    out_ref = torch.stack([ref.tree_attention(q, k, v, sl, tb["mask"]) for q, k, v in layers])
+    kd, vd = [l[1].to(DEV) for l in layers], [l[2].to(DEV) for l in layers]
+    k0, v0 = [t.clone() for t in kd], [t.clone() for t in vd]
+    hidden, W1, b1, W2, root = inp
+    a = binding.StepArgs()
+    a.B, a.H, a.V, a.Hq, a.Hkv, a.D, a.n_layers, a.Lcap = B, 256, 2000, 8, 2, 128, n_layers, Lcap
+    a.stride_b, a.stride_h, a.stride_t, a.scale = 2 * Lcap * 128, Lcap * 128, 128, 0.0
+    dev = dict(hidden=hidden.to(DEV), W1=W1.to(DEV), b1=b1.to(DEV), W2=W2.to(DEV), root_tok=root.to(DEV),
+               q_layers=torch.stack([l[0] for l in layers]).to(DEV), logits=logits.to(DEV), seq_lens=sl.to(DEV),
+               cand=_i32(B, tree.C), cand_logit=torch.zeros(B, tree.C - 1, device=DEV), tree_tok=_i32(B, T),
+               out_layers=torch.zeros(n_layers, B, T, 8, 128, dtype=torch.bfloat16, device=DEV),
+               accept_len=_i32(B), best_path=_i32(B), acc_nodes=_i32(B, K + 1), acc_tok=_i32(B, K + 1),
+               next_root=_i32(B), status=_i32(B), k_caches=binding.cache_pointer_array(kd, DEV),
+               v_caches=binding.cache_pointer_array(vd, DEV), k_caches_host=binding.cache_pointer_array(kd),
+               v_caches_host=binding.cache_pointer_array(vd), ws=workspace(tree, B, 256, 2000, 8, 2, 128, Lcap))
+    for name, t in dev.items():
+        setattr(a, name, t.data_ptr())
+    a.ws_bytes = dev["ws"].numel()
+    sl0 = sl.to(DEV)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        binding.mtv_verify_step(tree, a)             # once outside capture: first-use set-up happens here
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            binding.mtv_verify_step(tree, a)
+    for _ in range(2):                               # restore the inputs the step consumed, then replay
+        dev["seq_lens"].copy_(sl0)
+        for l in range(n_layers):
+            kd[l].copy_(k0[l]); vd[l].copy_(v0[l])
+        for n in ("tree_tok", "accept_len", "acc_nodes", "next_root"):
+            dev[n].fill_(-7)
+        dev["out_layers"].zero_()
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(dev["tree_tok"].cpu(), tt_ref)
+        for name in ("accept_len", "best_path", "acc_nodes", "acc_tok", "next_root"):
+            assert torch.equal(dev[name].cpu(), acc_ref[name]), name
+        assert torch.equal(dev["seq_lens"].cpu(), sl + acc_ref["accept_len"] + 1)
+        for l in range(n_layers):
+            assert_close(dev["out_layers"][l], out_ref[l], "layer %d" % l)
+    assert binding.mtv_device_error(tree) == 0
