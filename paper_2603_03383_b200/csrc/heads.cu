@@ -13,7 +13,9 @@ namespace mtv {
 
 constexpr int HEADS_THREADS = 256;
 constexpr int HEADS_WARPS = HEADS_THREADS / 32;
-constexpr int NB_MAX = 4;  // batch rows handled by one pass over the weights
+// one pass over the weights serves 1, 2, 4 or 8 batch rows:
+// batch rows per pass for a batch of B rows
+static inline int nb_for(int B) { return B == 1 ? 1 : B == 2 ? 2 : B <= 4 ? 4 : 8; }
 
 // vocabulary projection: 2 groups of 8 consumer warps + 1 producer warp
 constexpr int VT_GROUP_WARPS = 8;
@@ -27,7 +29,7 @@ constexpr uint32_t VT_SMEM_MAX = 226 * 1024;  // the opt-in limit minus room for
 // of stages, and the byte offsets of every region.
 struct VocabSmem {
     int rows_per_stage, n_stages, n_it;
-    uint32_t stage_bytes, ring_bytes, xs_off, lists_off, bars_off, total;
+    uint32_t stage_bytes, ring_bytes, xs_off, lists_off, zbuf_off, bars_off, total;
 };
 static VocabSmem vocab_smem_plan(int NB, int H, int ctas_per_head) {
     VocabSmem s;
@@ -36,7 +38,8 @@ static VocabSmem vocab_smem_plan(int NB, int H, int ctas_per_head) {
     const uint32_t xs_bytes = (uint32_t)NB * s.n_it * 64 * 16;
     const uint32_t lists_bytes = (uint32_t)VT_CONS_WARPS * NB * MTV_MAX_TOPK * 8;
     const uint32_t merge_bytes = (uint32_t)ctas_per_head * MTV_MAX_TOPK * 8;   // final merge reuses the ring
-    const uint32_t fixed = xs_bytes + lists_bytes + 256;
+    const uint32_t zbuf_bytes = NB > 1 ? VT_GROUPS * 2 * VT_GROUP_WARPS * 32 * 4 : 0;   // partial logits of the column parts
+    const uint32_t fixed = xs_bytes + lists_bytes + zbuf_bytes + 256;
     s.rows_per_stage = 0;
     for (int rs = VT_GROUP_WARPS; rs >= 1; rs /= 2) {
         const uint32_t sb = rs * row_bytes;
@@ -52,7 +55,8 @@ static VocabSmem vocab_smem_plan(int NB, int H, int ctas_per_head) {
     if (s.ring_bytes < merge_bytes) s.ring_bytes = (merge_bytes + 127) / 128 * 128;
     s.xs_off = (s.ring_bytes + 127) / 128 * 128;
     s.lists_off = s.xs_off + xs_bytes;
-    s.bars_off = s.lists_off + lists_bytes;
+    s.zbuf_off = s.lists_off + lists_bytes;
+    s.bars_off = s.zbuf_off + zbuf_bytes;
     s.total = s.bars_off + 256;
     if (s.total > VT_SMEM_MAX) s.total = 0;
     return s;
@@ -66,7 +70,7 @@ HeadsWs heads_ws_layout(const mtv_tree *t, int B, int H, int V) {
     if (per_head > max_useful) per_head = max_useful;
     if (per_head < 1) per_head = 1;
     w.ctas_per_head = per_head;
-    const int btiles = (B + NB_MAX - 1) / NB_MAX;
+    const int btiles = (B + nb_for(B) - 1) / nb_for(B);
     size_t off = 0;
     w.hprime_off = off;   off = align_up(off + (size_t)t->K * B * H * sizeof(float), 256);
     w.part_val_off = off; off = align_up(off + (size_t)t->K * B * per_head * MTV_MAX_TOPK * sizeof(float), 256);
@@ -98,6 +102,30 @@ __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
+}
+
+// Sum over the 32 lanes of N per-lane values at once (N a power of two <= 32): afterwards lane l holds
+// in v[0] the sum of value number l / (32 / N).  N - 1 + log2(32 / N) shuffles instead of 5 N.
+template <int N>
+__device__ __forceinline__ void warp_sum_scatter(float (&v)[N], int lane) {
+    int n = N;
+#pragma unroll
+    for (int bit = 16; bit >= 1; bit >>= 1) {
+        if (n > 1) {
+            n >>= 1;
+            const bool up = (lane & bit) != 0;
+#pragma unroll
+            for (int i = 0; i < N / 2; ++i) {
+                if (i < n) {
+                    const float send = up ? v[i] : v[i + n];
+                    const float keep = up ? v[i + n] : v[i];
+                    v[i] = keep + __shfl_xor_sync(0xffffffffu, send, bit);
+                }
+            }
+        } else {
+            v[0] += __shfl_xor_sync(0xffffffffu, v[0], bit);
+        }
+    }
 }
 
 // (value, id) ordering of the candidate lists: larger value first, equal values by smaller id.
@@ -183,7 +211,7 @@ struct VocabParams {
     int32_t *tree_tok;
     int32_t *dev_error;
     int rows_per_stage, n_stages, n_it;
-    uint32_t stage_bytes, xs_off, lists_off, bars_off;
+    uint32_t stage_bytes, xs_off, lists_off, zbuf_off, bars_off;
 };
 
 template <int NB>
@@ -252,6 +280,7 @@ heads_vocab_topk_kernel(const VocabParams p) {
         }
     } else {
         // ---- consumers
+        if constexpr (NB == 1) {
         const int group = warp / VT_GROUP_WARPS, wr = warp % VT_GROUP_WARPS;
         float *my_val = lval + (warp * NB) * MTV_MAX_TOPK;
         int32_t *my_idx = lidx + (warp * NB) * MTV_MAX_TOPK;
@@ -328,6 +357,90 @@ heads_vocab_topk_kernel(const VocabParams p) {
                     }
                 }
             }
+        }
+            } else {
+        // Several batch rows: every activation chunk read from shared memory must serve several weight
+        // rows, or shared-memory bandwidth, not HBM, sets the pace.  A group's eight warps split a stage
+        // into row blocks of R rows and column parts: warp (rb, cp) multiplies rows [R rb, R rb + R) by
+        // the batch rows over the iterations it = cp, cp + ncp, ...; the column parts' partial logits
+        // meet in shared memory and the warp with cp = 0 of each row block keeps the candidate lists.
+        constexpr int R = NB >= 4 ? 4 : 2;
+        constexpr int NV = R * NB;                       // logits per warp and stage
+        const int group = warp / VT_GROUP_WARPS, wr = warp % VT_GROUP_WARPS;
+        const int nrb = RS / R, ncp = VT_GROUP_WARPS / nrb;   // the host guarantees RS >= R
+        const int rb = wr % nrb, cp = wr / nrb;
+        float *zbuf = reinterpret_cast<float *>(smem + p.zbuf_off) + group * 2 * VT_GROUP_WARPS * 32;   // [2][8 warps][32]
+        float *my_val = lval + (warp * NB) * MTV_MAX_TOPK;
+        int32_t *my_idx = lidx + (warp * NB) * MTV_MAX_TOPK;
+        bool ok = true;   // a warp whose wait ran out keeps the group barrier matched without waiting again
+        for (int t = group; t < n_chunks; t += VT_GROUPS) {
+            const int s = t % NST, use = t / NST;
+            if (*abort_flag) ok = false;
+            if (ok && use > 0) ok = ptx::mbar_wait(bars + (NST + s) * 8, (use - 1) & 1);   // see the single-row path
+            if (ok) ok = ptx::mbar_wait(bars + s * 8, use & 1);
+            if (!ok) *abort_flag = 1;
+            const int v0 = v_begin + t * RS;
+            const int rows = min(RS, v_end - v0);
+            float acc[NV];
+#pragma unroll
+            for (int i = 0; i < NV; ++i) acc[i] = 0.f;
+            const unsigned char *wblock = smem + s * p.stage_bytes + (size_t)(rb * R) * row_bytes;
+            for (int it = cp; it < p.n_it; it += ncp) {
+                const int c = it * 32 + lane;
+                if (c < n_chunk16) {
+                    float wf[R][8];
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+                        bf16x8_to_float(reinterpret_cast<const uint4 *>(wblock + (size_t)r * row_bytes)[c], wf[r]);
+#pragma unroll
+                    for (int b = 0; b < NB; ++b) {
+                        const float4 x0 = xs4[((b * p.n_it + it) * 2) * 32 + lane];
+                        const float4 x1 = xs4[((b * p.n_it + it) * 2 + 1) * 32 + lane];
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
+                            float a = acc[r * NB + b];
+                            a = fmaf(wf[r][0], x0.x, a); a = fmaf(wf[r][1], x0.y, a);
+                            a = fmaf(wf[r][2], x0.z, a); a = fmaf(wf[r][3], x0.w, a);
+                            a = fmaf(wf[r][4], x1.x, a); a = fmaf(wf[r][5], x1.y, a);
+                            a = fmaf(wf[r][6], x1.z, a); a = fmaf(wf[r][7], x1.w, a);
+                            acc[r * NB + b] = a;
+                        }
+                    }
+                }
+            }
+            warp_sum_scatter<NV>(acc, lane);   // lane l: partial logit number l / (32 / NV) of this column part
+            // every lane's reads of the stage are complete (their values fed the sums): release it
+            if (ok && lane == 0) ptx::mbar_arrive(bars + (NST + s) * 8);
+            float *zb = zbuf + ((t / VT_GROUPS) & 1) * VT_GROUP_WARPS * 32;
+            if (lane % (32 / NV) == 0) zb[wr * 32 + lane / (32 / NV)] = acc[0];
+            asm volatile("bar.sync %0, 256;" ::"r"(2 + group) : "memory");
+            if (cp == 0) {
+                // lane l < NV: row r = l / NB of the block, batch row b = l % NB
+                const int r = lane / NB, b = lane % NB;
+                float z = 0.f;
+                if (lane < NV)
+                    for (int q = 0; q < ncp; ++q) z += zb[(q * nrb + rb) * 32 + lane];
+                const int v = v0 + rb * R + r;
+                const bool live = lane < NV && rb * R + r < rows && b0 + b < p.B;
+#pragma unroll 1
+                for (int rr = 0; rr < R; ++rr) {
+                    if (live && r == rr &&
+                        cand_before(z, v, my_val[b * MTV_MAX_TOPK + kd - 1], my_idx[b * MTV_MAX_TOPK + kd - 1])) {
+                        // this lane is the only one that touches list b now: insertion into the sorted list
+                        int pos = kd - 1;
+                        while (pos > 0 && cand_before(z, v, my_val[b * MTV_MAX_TOPK + pos - 1],
+                                                      my_idx[b * MTV_MAX_TOPK + pos - 1])) {
+                            my_val[b * MTV_MAX_TOPK + pos] = my_val[b * MTV_MAX_TOPK + pos - 1];
+                            my_idx[b * MTV_MAX_TOPK + pos] = my_idx[b * MTV_MAX_TOPK + pos - 1];
+                            --pos;
+                        }
+                        my_val[b * MTV_MAX_TOPK + pos] = z;
+                        my_idx[b * MTV_MAX_TOPK + pos] = v;
+                    }
+                    __syncwarp();
+                }
+            }
+        }
         }
     }
     __syncthreads();
@@ -422,6 +535,7 @@ static int launch_heads(const mtv_tree *t, int B, int H, int V, const __nv_bfloa
     const size_t sm1 = (size_t)NB * H * sizeof(float);
     const VocabSmem S = vocab_smem_plan(NB, H, L.ctas_per_head);
     if (sm1 > VT_SMEM_MAX || S.total == 0) return MTV_ERR_UNSUPPORTED_SHAPE;
+    if (NB > 1 && S.rows_per_stage < (NB >= 4 ? 4 : 2)) return MTV_ERR_UNSUPPORTED_SHAPE;   // rows too long for a block of rows per stage
     static bool attr_done = false;
     if (!attr_done) {
         MTV_CUDA_CHECK(cudaFuncSetAttribute(heads_resblock_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, VT_SMEM_MAX));
@@ -447,7 +561,7 @@ static int launch_heads(const mtv_tree *t, int B, int H, int V, const __nv_bfloa
     p.cand = cand; p.cand_logit = cand_logit; p.tree_tok = tree_tok;
     p.dev_error = t->d_error;
     p.rows_per_stage = S.rows_per_stage; p.n_stages = S.n_stages; p.n_it = S.n_it;
-    p.stage_bytes = S.stage_bytes; p.xs_off = S.xs_off; p.lists_off = S.lists_off; p.bars_off = S.bars_off;
+    p.stage_bytes = S.stage_bytes; p.xs_off = S.xs_off; p.lists_off = S.lists_off; p.zbuf_off = S.zbuf_off; p.bars_off = S.bars_off;
     {
         TapScope tap(MTV_KERNEL_HEADS_VOCAB_TOPK, st);
         heads_vocab_topk_kernel<NB><<<dim3(L.ctas_per_head, t->K, btiles), VT_THREADS, S.total, st>>>(p);
@@ -480,7 +594,8 @@ extern "C" int medusa_heads_topk(const mtv_tree_t *tree, int B, int H, int V,
     int rc;
     if (B == 1) rc = launch_heads<1>(tree, B, H, V, h, w1, bb, w2, root_tok, cand, cand_logit, tree_tok, L, (char *)ws, st);
     else if (B == 2) rc = launch_heads<2>(tree, B, H, V, h, w1, bb, w2, root_tok, cand, cand_logit, tree_tok, L, (char *)ws, st);
-    else rc = launch_heads<NB_MAX>(tree, B, H, V, h, w1, bb, w2, root_tok, cand, cand_logit, tree_tok, L, (char *)ws, st);
+    else if (B <= 4) rc = launch_heads<4>(tree, B, H, V, h, w1, bb, w2, root_tok, cand, cand_logit, tree_tok, L, (char *)ws, st);
+    else rc = launch_heads<8>(tree, B, H, V, h, w1, bb, w2, root_tok, cand, cand_logit, tree_tok, L, (char *)ws, st);
     if (rc != MTV_OK) return rc;
     MTV_CUDA_CHECK(cudaGetLastError());
     return MTV_OK;
