@@ -40,6 +40,9 @@ def parse():
     ap.add_argument("--no-taps", action="store_true", help="skip per-kernel event timing")
     ap.add_argument("--launch", default="graph", choices=["graph", "stream"],
                     help="timed steps: replay of one captured CUDA graph per step, or plain stream launches")
+    ap.add_argument("--overhead-sweep", action="store_true",
+                    help="instead of the step benchmark: time tree attention (T nodes) against single-token decode "
+                         "attention (a root-only tree) over prefix lengths, the attention part of the paper's overhead ratio")
     return ap.parse_args()
 
 
@@ -489,8 +492,52 @@ def run_reference(args):
     }))
 
 
+def run_overhead_sweep(args):
+    """Attention part of the paper's Overhead = Time_speculative / Time_autoregressive (Eq. 3) on this GPU:
+    the T-node tree attention call against the same call with a root-only tree (one query token), per
+    prefix length, on 32 rotating KV caches.  One JSON line per length."""
+    import torch
+    from paper_2603_03383_b200 import binding, synth
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    w = synth.WORKLOADS["long"]
+    nodes = binding.tree_gen_rank_prior(w.K, w.T, w.R_max)
+    trees = {"tree": binding.tree_build_static(w.K, nodes), "single": binding.tree_build_static(w.K, [])}
+    layers, reps = 32, 5
+    for L in (128, 512, 1024, 2048, 4096, 8192, 16384, 32768):
+        res = {}
+        for name, tree in trees.items():
+            T = tree.T
+            Lcap = L + T
+            qs = [synth.normal_bf16(7, synth.TID_Q + l, (1, T, w.Hq, w.D), device=dev) for l in range(layers)]
+            ks = [synth.normal_bf16(7, synth.TID_K + l, (1, w.Hkv, Lcap, w.D), device=dev) for l in range(layers)]
+            vs = [synth.normal_bf16(7, synth.TID_V + l, (1, w.Hkv, Lcap, w.D), device=dev) for l in range(layers)]
+            out = torch.zeros_like(qs[0])
+            sl = torch.tensor([L], dtype=torch.int32, device=dev)
+            ws = torch.empty(binding.mtv_workspace_bytes(tree, 1, 0, 0, w.Hq, w.Hkv, w.D, Lcap), dtype=torch.uint8,
+                             device=dev)
+            for l in range(layers):
+                binding.tree_verify_attention(tree, qs[l], ks[l], vs[l], sl, out, ws)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                for l in range(layers):
+                    binding.tree_verify_attention(tree, qs[l], ks[l], vs[l], sl, out, ws)
+            e1.record()
+            torch.cuda.synchronize()
+            res[name] = e0.elapsed_time(e1) * 1e3 / (reps * layers)
+            del qs, ks, vs
+        print(json.dumps({"prefix": L, "tree_nodes": trees["tree"].T, "us_tree_attention": res["tree"],
+                          "us_single_token_attention": res["single"],
+                          "attention_overhead_ratio": res["tree"] / res["single"]}))
+
+
 if __name__ == "__main__":
     a = parse()
+    if a.overhead_sweep:
+        run_overhead_sweep(a)
+        sys.exit(0)
     if a.impl == "reference":
         run_reference(a)
     else:
