@@ -329,6 +329,7 @@ def run_ours(args):
         "e2e": {"value": world / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps},
         "gpu_launches": K_steps * LAUNCHES_PER_STEP(n_layers),
+        "device_error": binding.mtv_device_error(tree, clear=False),
         "step_roofline": {"algorithmic_bytes": alg["step"], "achieved_gbs": alg["step"] / ms_step / 1e6,
                           "frac_of_measured": alg["step"] / ms_step / 1e6 / pk["hbm_gbs"],
                           "frac_of_8tbs": alg["step"] / ms_step / 1e6 / 8000.0},
