@@ -132,6 +132,23 @@ int medusa_heads_topk(const mtv_tree_t *tree, int B, int H, int V,
                       void *ws, size_t ws_bytes, void *stream);
 
 /* ---------------------------------------------------------------------------
+ * Tree K/V append with rotary embedding — the step just before the tree attention; Section 3.2
+ * ("Tensorization of Tree Topology": tree_indices maps the flattened nodes to their positions).
+ * For sequence b and node i, position = seq_lens[b] + depth[i]:
+ *   angle_d = position * theta^(-2d/D), d < D/2        (rotate-half pairing, a reading: the paper is silent)
+ *   (x[d], x[d + D/2]) -> (x[d] cos - x[d + D/2] sin, x[d + D/2] cos + x[d] sin)
+ * q [B][T][Hq][D] is rotated in place; k_new, v_new [B][T][Hkv][D]: the rotated K row and the V row
+ * are written to cache row seq_lens[b] + i (cache layout and strides as in tree_verify_attention).
+ * Angles in double precision, arithmetic in fp32, bf16 results (round to nearest even).
+ * All pointers device.  rope_theta == 0 means 10000.  status[b] = MTV_ERR_CAPACITY (nothing
+ * written for b) if seq_lens[b] + T > Lcap.  seq_lens is not changed.
+ */
+int tree_kv_append_rope(const mtv_tree_t *tree, int B, int Hq, int Hkv, int D, mtv_bf16 *q,
+                        const mtv_bf16 *k_new, const mtv_bf16 *v_new, mtv_bf16 *k_cache, mtv_bf16 *v_cache,
+                        int64_t stride_b, int64_t stride_h, int64_t stride_t, int Lcap,
+                        const int32_t *seq_lens, float rope_theta, int32_t *status, void *stream);
+
+/* ---------------------------------------------------------------------------
  * Tree attention — Section 3.2 / Fig. 2(b): the T tree nodes attend to the KV cache
  * under the static visibility matrix.  For sequence b, node i, query head h
  * (KV head g = h / (Hq/Hkv)):

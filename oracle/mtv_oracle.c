@@ -256,3 +256,38 @@ void mtv_ref_kv_compact(int B, int Hkv, int D,
                        (size_t)D * sizeof(uint16_t));
             }
 }
+
+/* ------------------------------------------------------ tree K/V append + RoPE
+ * The step just before the tree attention (Section 3.2: tree_indices maps the flattened tree
+ * nodes to their positions): node i of sequence b sits at position seq_lens[b] + depth[i] and
+ * its K / V rows go to cache row seq_lens[b] + i.  Rotary embedding in the rotate-half pairing:
+ * for d < D/2, angle = position * theta^(-2d/D),
+ *     (x[d], x[d + D/2]) -> (x[d] cos - x[d + D/2] sin,  x[d + D/2] cos + x[d] sin).
+ * q [B][T][Hq][D] and k_new, v_new [B][T][Hkv][D] are bf16; the rotated q and k come back as
+ * doubles (q_out [B][T][Hq][D], k_out [B][T][Hkv][D]); V is copied unchanged by the caller.
+ */
+void mtv_ref_rope(int B, int T, int Hq, int Hkv, int D,
+                  const uint16_t *q, const uint16_t *k_new, const int32_t *seq_lens, const int32_t *depth,
+                  double theta, double *q_out, double *k_out)
+{
+    const int half = D / 2;
+    for (int b = 0; b < B; ++b)
+        for (int i = 0; i < T; ++i) {
+            const double pos = (double)seq_lens[b] + (double)depth[i];
+            for (int which = 0; which < 2; ++which) {
+                const int Hn = which ? Hkv : Hq;
+                const uint16_t *src = which ? k_new : q;
+                double *dst = which ? k_out : q_out;
+                for (int h = 0; h < Hn; ++h) {
+                    const size_t base = (((size_t)b * T + i) * Hn + h) * D;
+                    for (int d = 0; d < half; ++d) {
+                        const double ang = pos * pow(theta, -2.0 * d / D);
+                        const double c = cos(ang), sn = sin(ang);
+                        const double x1 = bf16_to_double(src[base + d]), x2 = bf16_to_double(src[base + d + half]);
+                        dst[base + d] = x1 * c - x2 * sn;
+                        dst[base + d + half] = x2 * c + x1 * sn;
+                    }
+                }
+            }
+        }
+}

@@ -151,3 +151,17 @@ def kv_compact(cache, seq_lens, accept_len, acc_nodes):
                              C.c_int64(sb), C.c_int64(sh), C.c_int64(st),
                              _p(seq_lens), _p(accept_len), _p(acc_nodes), K)
     return dst, seq_lens + accept_len + 1
+
+
+def rope(q, k_new, seq_lens, depth, theta=10000.0):
+    """Rotary embedding of the tree nodes' q [B,T,Hq,D] and k_new [B,T,Hkv,D] at positions seq_lens[b] + depth[i]
+    (rotate-half pairing) -> (q_out, k_out) float64."""
+    B, T, Hq, D = q.shape
+    Hkv = k_new.shape[2]
+    q, k_new = q.contiguous(), k_new.contiguous()
+    seq_lens, depth = _i32(seq_lens), _i32(depth)
+    q_out = torch.empty(B, T, Hq, D, dtype=torch.float64)
+    k_out = torch.empty(B, T, Hkv, D, dtype=torch.float64)
+    lib().mtv_ref_rope(B, T, Hq, Hkv, D, _p(q), _p(k_new), _p(seq_lens), _p(depth), C.c_double(theta), _p(q_out),
+                       _p(k_out))
+    return q_out, k_out

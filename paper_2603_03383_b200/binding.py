@@ -26,7 +26,7 @@ EXPORTS = ["tree_build_static", "tree_gen_cartesian", "tree_gen_rank_prior", "tr
            "mtv_workspace_bytes", "medusa_heads_topk", "tree_verify_attention", "tree_accept",
            "kv_compact_accepted", "mtv_verify_step", "mtv_verify_step_host", "mtv_last_error",
            "mtv_set_kernel_taps", "mtv_kernel_taps_used", "mtv_device_error",
-           "tree_accept_static_scratch", "tree_accept_static_scratch_capacity"]
+           "tree_accept_static_scratch", "tree_accept_static_scratch_capacity", "tree_kv_append_rope"]
 
 
 class MtvError(RuntimeError):
@@ -98,6 +98,8 @@ def lib():
         L.mtv_device_error.argtypes = [vp, i32, C.POINTER(C.c_int32)]
         L.tree_accept_static_scratch.argtypes = [vp, i32, i32] + [vp] * 7 + [vp]
         L.tree_accept_static_scratch_capacity.restype = sz
+        L.tree_kv_append_rope.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, i64, i64, i64, i32, vp, C.c_float,
+                                          vp, vp]
         _lib = L
     return _lib
 
@@ -207,6 +209,18 @@ def tree_verify_attention(tree, q, k_cache, v_cache, seq_lens, out, ws, scale=0.
     _check(lib().tree_verify_attention(tree.handle, B, Hq, Hkv, D, _ptr(q), _ptr(k_cache), _ptr(v_cache),
                                        sb, sh, st, Lcap, _ptr(seq_lens), scale, _ptr(out), _ptr(status), p, n,
                                        _stream(stream)), "tree_verify_attention")
+
+
+def tree_kv_append_rope(tree, q, k_new, v_new, k_cache, v_cache, seq_lens, rope_theta=0.0, status=None, stream=None,
+                        Lcap=None):
+    B, T, Hq, D = q.shape
+    Hkv = k_new.shape[2]
+    Lcap = k_cache.shape[2] if Lcap is None else Lcap
+    sb, sh, st = k_cache.stride(0), k_cache.stride(1), k_cache.stride(2)
+    assert (v_cache.stride(0), v_cache.stride(1), v_cache.stride(2)) == (sb, sh, st)
+    _check(lib().tree_kv_append_rope(tree.handle, B, Hq, Hkv, D, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache),
+                                     _ptr(v_cache), sb, sh, st, Lcap, _ptr(seq_lens), rope_theta, _ptr(status),
+                                     _stream(stream)), "tree_kv_append_rope")
 
 
 def tree_accept(tree, logits, tree_tok, accept_len, best_path, acc_nodes, acc_tok, next_root, ws, stream=None):

@@ -26,6 +26,7 @@ struct mtv_tree {
     const int32_t *d_kd = nullptr;            // [K]
     const int32_t *d_cand_offset = nullptr;   // [K]
     int32_t *d_error = nullptr;               // sticky device-side error word (0 = none)
+    const int32_t *d_depth = nullptr;         // [T]
     int32_t *d_counters = nullptr;            // [512] merge counters of the attention kernel, zero between calls
 };
 

@@ -137,7 +137,7 @@ extern "C" int tree_build_static(int K, int n_nodes, const int32_t *node_ranks, 
     if (upload) {
         const size_t n_ti = T, n_ri = (size_t)tr->P * (K + 1), n_anc = (size_t)T * 2;
         size_t o_ti = 0, o_ri = mtv::align_up(o_ti + n_ti * 4, 16), o_anc = mtv::align_up(o_ri + n_ri * 4, 16);
-        size_t o_kd = o_anc + n_anc * 8, o_co = o_kd + MTV_MAX_K * 4, o_err = o_co + MTV_MAX_K * 4, o_cnt = o_err + 16, total = o_cnt + 512 * 4;
+        size_t o_kd = o_anc + n_anc * 8, o_co = o_kd + MTV_MAX_K * 4, o_err = o_co + MTV_MAX_K * 4, o_cnt = o_err + 16, o_dep = o_cnt + 512 * 4, total = o_dep + (size_t)T * 4;
         std::vector<unsigned char> blob(total, 0);
         memcpy(blob.data() + o_ti, tr->tree_indices.data(), n_ti * 4);
         memcpy(blob.data() + o_ri, tr->retrieve.data(), n_ri * 4);
@@ -146,6 +146,7 @@ extern "C" int tree_build_static(int K, int n_nodes, const int32_t *node_ranks, 
                 memcpy(blob.data() + o_anc + ((size_t)i * 2 + w) * 8, &tr->anc[(size_t)i * tr->anc_words + w], 8);
         memcpy(blob.data() + o_kd, tr->k_d, MTV_MAX_K * 4);
         memcpy(blob.data() + o_co, tr->cand_offset, MTV_MAX_K * 4);
+        memcpy(blob.data() + o_dep, tr->depth.data(), (size_t)T * 4);
         cudaError_t e = cudaGetDevice(&tr->device);
         if (e == cudaSuccess) e = cudaMalloc(&tr->d_blob, total);
         if (e == cudaSuccess) e = cudaMemcpy(tr->d_blob, blob.data(), total, cudaMemcpyHostToDevice);
@@ -163,6 +164,7 @@ extern "C" int tree_build_static(int K, int n_nodes, const int32_t *node_ranks, 
         tr->d_cand_offset = (const int32_t *)(base + o_co);
         tr->d_error = (int32_t *)(base + o_err);
         tr->d_counters = (int32_t *)(base + o_cnt);
+        tr->d_depth = (const int32_t *)(base + o_dep);
         tr->on_device = true;
     }
     *out = tr;

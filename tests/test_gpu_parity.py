@@ -386,3 +386,47 @@ def test_full_step_replays_from_a_cuda_graph():
         for l in range(n_layers):
             assert_close(dev["out_layers"][l], out_ref[l], "layer %d" % l)
     assert binding.mtv_device_error(tree) == 0
+
+
+# ------------------------------------------------------------ append + RoPE
+@pytest.mark.parametrize("Hq,Hkv,D,lens,theta", [(32, 8, 128, [8192], 0.0), (8, 2, 64, [0, 517, 30000], 500000.0)])
+def test_tree_kv_append_rope(Hq, Hkv, D, lens, theta):
+    tb, tree = make_tree("rank_prior", 4, (), 64)
+    T, B = tree.T, len(lens)
+    Lcap = max(lens) + T + 3
+    q = synth.normal_bf16(5, 1, (B, T, Hq, D))
+    k_new = synth.normal_bf16(5, 2, (B, T, Hkv, D))
+    v_new = synth.normal_bf16(5, 3, (B, T, Hkv, D))
+    kc = synth.normal_bf16(5, 4, (B, Hkv, Lcap, D))
+    vc = synth.normal_bf16(5, 5, (B, Hkv, Lcap, D))
+    q_ref, k_ref = ref.rope(q, k_new, lens, tb["depth"], theta or 10000.0)
+    qd, kd, vd = q.to(DEV), kc.to(DEV), vc.to(DEV)
+    status = _i32(B)
+    sl = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    binding.tree_kv_append_rope(tree, qd, k_new.to(DEV), v_new.to(DEV), kd, vd, sl, rope_theta=theta, status=status)
+    torch.cuda.synchronize()
+    assert status.tolist() == [0] * B and sl.cpu().tolist() == lens
+    assert_close(qd, q_ref, "rotated q")
+    # one bf16 rounding of an fp32 result whose angle came from double precision: within an ulp of the checker
+    assert (qd.double().cpu() - q_ref).abs().max().item() <= 2.0 ** -7 * q_ref.abs().max().item()
+    for b, L in enumerate(lens):
+        got_k = kd[b, :, L:L + T].cpu().permute(1, 0, 2)            # [T][Hkv][D]
+        assert_close(got_k, k_ref[b], "rotated k in the cache")
+        assert torch.equal(vd[b, :, L:L + T].cpu().permute(1, 0, 2), v_new[b])          # V copied bit-exactly
+        assert torch.equal(kd[b, :, :L].cpu(), kc[b, :, :L]) and torch.equal(kd[b, :, L + T:].cpu(), kc[b, :, L + T:])
+        assert torch.equal(vd[b, :, :L].cpu(), vc[b, :, :L]) and torch.equal(vd[b, :, L + T:].cpu(), vc[b, :, L + T:])
+
+
+def test_tree_kv_append_rope_capacity():
+    tb, tree = make_tree("cartesian", 2, (2, 2))
+    T, B, Lcap = tree.T, 2, 20
+    q = synth.normal_bf16(6, 1, (B, T, 4, 64), device=DEV)
+    q0 = q.clone()
+    kn, vn = synth.normal_bf16(6, 2, (B, T, 2, 64), device=DEV), synth.normal_bf16(6, 3, (B, T, 2, 64), device=DEV)
+    kc, vc = torch.zeros(B, 2, Lcap, 64, dtype=torch.bfloat16, device=DEV), torch.zeros(B, 2, Lcap, 64, dtype=torch.bfloat16, device=DEV)
+    status = _i32(B)
+    binding.tree_kv_append_rope(tree, q, kn, vn, kc, vc, torch.tensor([Lcap - T + 1, 3], dtype=torch.int32, device=DEV),
+                                status=status)
+    torch.cuda.synchronize()
+    assert status.tolist() == [binding.MTV_ERR_CAPACITY, 0]
+    assert torch.equal(q[0], q0[0]) and not torch.equal(q[1], q0[1]) and bool((kc[0] == 0).all())
