@@ -95,3 +95,45 @@ def test_accept_full_size(name):
     torch.cuda.synchronize()
     for name_, t in outs.items():
         assert torch.equal(t.cpu(), want[name_]), name_
+
+
+@pytest.mark.parametrize("name,reps", [("long", 300), ("short", 300), ("stress", 20)])
+def test_attention_is_bitwise_repeatable(name, reps):
+    """The key splits of a query block meet through counters and bulk copies inside one launch; the merge order
+    is fixed, so repeated calls must give bit-identical output.  A missing fence in that exchange would show up
+    here as a rare difference."""
+    w = synth.WORKLOADS[name]
+    tb, tree = workload_tree(w)
+    T, B = tree.T, w.B
+    lens = synth.seq_lens(w).to(DEV)
+    Lcap = int(w.L_hi) + T
+    q, k, v = synth.attention_inputs(B, T, w.Hq, w.Hkv, w.D, Lcap, w.seed + 5, device=DEV)
+    ws = workspace(tree, B, 0, 0, w.Hq, w.Hkv, w.D, Lcap)
+    first = torch.zeros(B, T, w.Hq, w.D, dtype=torch.bfloat16, device=DEV)
+    binding.tree_verify_attention(tree, q, k, v, lens, first, ws)
+    outs = [torch.zeros_like(first) for _ in range(4)]
+    bad = torch.zeros((), dtype=torch.int64, device=DEV)
+    for i in range(reps):
+        o = outs[i % 4]
+        o.fill_(float("nan"))
+        binding.tree_verify_attention(tree, q, k, v, lens, o, ws)
+        bad += (o.view(torch.int16) != first.view(torch.int16)).sum()
+    torch.cuda.synchronize()
+    assert binding.mtv_device_error(tree) == 0
+    assert int(bad) == 0
+
+
+def test_heads_are_bitwise_repeatable():
+    w = synth.WORKLOADS["long"]
+    tb, tree = workload_tree(w)
+    hidden, W1, b1, W2, root = synth.head_inputs(4, w.H, 32768, w.K, 99, device=DEV)    # the 4-row (blocked) path
+    ws = workspace(tree, 4, w.H, 32768, 0, 0, 0, 0)
+    ref_c = torch.zeros(4, tree.C, dtype=torch.int32, device=DEV)
+    ref_l = torch.zeros(4, tree.C - 1, device=DEV)
+    tt = torch.zeros(4, tree.T, dtype=torch.int32, device=DEV)
+    binding.medusa_heads_topk(tree, hidden, W1, b1, W2, root, ref_c, ref_l, tt, ws)
+    for _ in range(30):
+        c, l = torch.zeros_like(ref_c), torch.zeros_like(ref_l)
+        binding.medusa_heads_topk(tree, hidden, W1, b1, W2, root, c, l, tt, ws)
+        assert torch.equal(c, ref_c) and torch.equal(l, ref_l)
+    assert binding.mtv_device_error(tree) == 0
