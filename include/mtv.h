@@ -254,11 +254,16 @@ int mtv_verify_step(const mtv_tree_t *tree, const mtv_step_args *args, void *str
 
 /* The same step for a caller whose per-step tensors live in (pinned) host memory.
  * Copies hidden, root_tok, q_layers and logits host->device into the device
- * buffers named in `dev`, runs mtv_verify_step, copies tree_tok, out_layers,
+ * buffers named in `dev`, runs the step, copies tree_tok, out_layers,
  * accept_len, best_path, acc_nodes, acc_tok, next_root and seq_lens back to the
  * host buffers, and synchronises the stream before returning.  Weights, KV caches
  * and the tree stay resident on the device.  `host` uses the same struct: only
- * the fields listed above are read from it. */
+ * the fields listed above are read from it.
+ * The transfers overlap the compute on two copy streams that the library creates
+ * on first use: queries and logits go up while the heads run, the attention
+ * outputs come down in groups of layers while later layers run.  Unlike the other
+ * step calls this one is therefore neither allocation-free on its first call nor
+ * capturable; use pinned host buffers, or the copies serialise. */
 int mtv_verify_step_host(const mtv_tree_t *tree, const mtv_step_args *dev, const mtv_step_args *host,
                          void *stream);
 

@@ -34,26 +34,88 @@ extern "C" int mtv_verify_step(const mtv_tree_t *tree, const mtv_step_args *a, v
                                stream);
 }
 
+namespace {
+// Copy streams and events of the host-buffer variant, created on first use (one set per process;
+// the variant synchronises anyway, so it is not one of the allocation-free hot calls).
+struct HostStepAux {
+    cudaStream_t up = nullptr, down = nullptr;
+    cudaEvent_t start = nullptr, q_up = nullptr, logits_up = nullptr, down_done = nullptr;
+    cudaEvent_t chunk[4] = {nullptr, nullptr, nullptr, nullptr};
+    bool ready = false;
+};
+HostStepAux g_aux;
+int host_step_aux() {
+    if (g_aux.ready) return MTV_OK;
+    MTV_CUDA_CHECK(cudaStreamCreateWithFlags(&g_aux.up, cudaStreamNonBlocking));
+    MTV_CUDA_CHECK(cudaStreamCreateWithFlags(&g_aux.down, cudaStreamNonBlocking));
+    cudaEvent_t *ev[] = {&g_aux.start, &g_aux.q_up, &g_aux.logits_up, &g_aux.down_done, &g_aux.chunk[0], &g_aux.chunk[1],
+                         &g_aux.chunk[2], &g_aux.chunk[3]};
+    for (cudaEvent_t *e : ev) MTV_CUDA_CHECK(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
+    g_aux.ready = true;
+    return MTV_OK;
+}
+}  // namespace
+
+// The transfers overlap the compute: the queries and the base-model logits go up on a copy stream while the
+// heads run (attention waits for the queries, acceptance for the logits), and the attention outputs come
+// down on a second copy stream in up to four groups of layers while later layers are still running.
 extern "C" int mtv_verify_step_host(const mtv_tree_t *tree, const mtv_step_args *d, const mtv_step_args *h,
                                     void *stream) {
-    if (!tree || !d || !h) return MTV_ERR_INVALID_ARG;
-    cudaStream_t st = (cudaStream_t)stream;
+    if (!tree || !d || !h || !d->k_caches_host || !d->v_caches_host) return MTV_ERR_INVALID_ARG;
+    if (host_step_aux() != MTV_OK) return MTV_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream, up = g_aux.up, down = g_aux.down;
     const size_t B = d->B, T = tree->T, K = tree->K;
-    const size_t q_bytes = (size_t)d->n_layers * B * T * d->Hq * d->D * 2;
+    const size_t per_layer = B * T * d->Hq * d->D;           // elements
+    const size_t q_bytes = (size_t)d->n_layers * per_layer * 2;
+    // uploads
+    MTV_CUDA_CHECK(cudaEventRecord(g_aux.start, st));         // the copy streams start where the caller's stream is
+    MTV_CUDA_CHECK(cudaStreamWaitEvent(up, g_aux.start, 0));
+    MTV_CUDA_CHECK(cudaStreamWaitEvent(down, g_aux.start, 0));
     MTV_CUDA_CHECK(cudaMemcpyAsync((void *)d->hidden, h->hidden, B * d->H * 2, cudaMemcpyHostToDevice, st));
     MTV_CUDA_CHECK(cudaMemcpyAsync((void *)d->root_tok, h->root_tok, B * 4, cudaMemcpyHostToDevice, st));
-    MTV_CUDA_CHECK(cudaMemcpyAsync((void *)d->q_layers, h->q_layers, q_bytes, cudaMemcpyHostToDevice, st));
-    MTV_CUDA_CHECK(cudaMemcpyAsync((void *)d->logits, h->logits, B * T * d->V * 2, cudaMemcpyHostToDevice, st));
-    int rc = mtv_verify_step(tree, d, stream);
+    MTV_CUDA_CHECK(cudaMemcpyAsync((void *)d->q_layers, h->q_layers, q_bytes, cudaMemcpyHostToDevice, up));
+    MTV_CUDA_CHECK(cudaEventRecord(g_aux.q_up, up));
+    MTV_CUDA_CHECK(cudaMemcpyAsync((void *)d->logits, h->logits, B * T * d->V * 2, cudaMemcpyHostToDevice, up));
+    MTV_CUDA_CHECK(cudaEventRecord(g_aux.logits_up, up));
+    // heads
+    int rc = medusa_heads_topk(tree, d->B, d->H, d->V, d->hidden, d->W1, d->b1, d->W2, d->root_tok, d->cand, d->cand_logit,
+                               d->tree_tok, d->ws, d->ws_bytes, stream);
     if (rc != MTV_OK) return rc;
     MTV_CUDA_CHECK(cudaMemcpyAsync(h->tree_tok, d->tree_tok, B * T * 4, cudaMemcpyDeviceToHost, st));
-    MTV_CUDA_CHECK(cudaMemcpyAsync(h->out_layers, d->out_layers, q_bytes, cudaMemcpyDeviceToHost, st));
+    // attention, its outputs leaving in groups of layers
+    MTV_CUDA_CHECK(cudaStreamWaitEvent(st, g_aux.q_up, 0));
+    const int per_group = (d->n_layers + 3) / 4;
+    int sent = 0, n_sent = 0;
+    for (int l = 0; l < d->n_layers; ++l) {
+        rc = tree_verify_attention(tree, d->B, d->Hq, d->Hkv, d->D, d->q_layers + l * per_layer, d->k_caches_host[l],
+                                   d->v_caches_host[l], d->stride_b, d->stride_h, d->stride_t, d->Lcap, d->seq_lens,
+                                   d->scale, d->out_layers + l * per_layer, d->status, d->ws, d->ws_bytes, stream);
+        if (rc != MTV_OK) return rc;
+        if ((l + 1) % per_group == 0 || l + 1 == d->n_layers) {
+            cudaEvent_t ev = g_aux.chunk[n_sent++ % 4];
+            MTV_CUDA_CHECK(cudaEventRecord(ev, st));
+            MTV_CUDA_CHECK(cudaStreamWaitEvent(down, ev, 0));
+            MTV_CUDA_CHECK(cudaMemcpyAsync(h->out_layers + sent * per_layer, d->out_layers + sent * per_layer,
+                                           (size_t)(l + 1 - sent) * per_layer * 2, cudaMemcpyDeviceToHost, down));
+            sent = l + 1;
+        }
+    }
+    // acceptance and compaction
+    MTV_CUDA_CHECK(cudaStreamWaitEvent(st, g_aux.logits_up, 0));
+    rc = tree_accept(tree, d->B, d->V, d->logits, d->tree_tok, d->accept_len, d->best_path, d->acc_nodes, d->acc_tok,
+                     d->next_root, d->ws, d->ws_bytes, stream);
+    if (rc != MTV_OK) return rc;
+    rc = kv_compact_accepted(tree, d->B, d->Hkv, d->D, d->n_layers, d->k_caches, d->v_caches, d->stride_b, d->stride_h,
+                             d->stride_t, d->Lcap, d->seq_lens, d->accept_len, d->acc_nodes, d->status, stream);
+    if (rc != MTV_OK) return rc;
     MTV_CUDA_CHECK(cudaMemcpyAsync(h->accept_len, d->accept_len, B * 4, cudaMemcpyDeviceToHost, st));
     MTV_CUDA_CHECK(cudaMemcpyAsync(h->best_path, d->best_path, B * 4, cudaMemcpyDeviceToHost, st));
     MTV_CUDA_CHECK(cudaMemcpyAsync(h->acc_nodes, d->acc_nodes, B * (K + 1) * 4, cudaMemcpyDeviceToHost, st));
     MTV_CUDA_CHECK(cudaMemcpyAsync(h->acc_tok, d->acc_tok, B * (K + 1) * 4, cudaMemcpyDeviceToHost, st));
     MTV_CUDA_CHECK(cudaMemcpyAsync(h->next_root, d->next_root, B * 4, cudaMemcpyDeviceToHost, st));
     MTV_CUDA_CHECK(cudaMemcpyAsync(h->seq_lens, d->seq_lens, B * 4, cudaMemcpyDeviceToHost, st));
+    MTV_CUDA_CHECK(cudaEventRecord(g_aux.down_done, down));
+    MTV_CUDA_CHECK(cudaStreamWaitEvent(st, g_aux.down_done, 0));
     MTV_CUDA_CHECK(cudaStreamSynchronize(st));
     return MTV_OK;
 }
