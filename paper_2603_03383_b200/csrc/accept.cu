@@ -46,19 +46,31 @@ node_argmax_partial_kernel(int V, const __nv_bfloat16 *__restrict__ logits, unsi
     unsigned long long best = 0;
     const bool aligned = (((size_t)row * V) % 8) == 0;
     if (aligned) {
-        for (int i = begin + threadIdx.x * 8; i < end; i += ARGMAX_THREADS * 8) {
-            if (i + 8 <= end) {
-                uint4 u;
-                asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                             : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w) : "l"(p + i));
-                const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+        // four independent 16-byte loads in flight per thread, then the (cheap) key arithmetic
+        constexpr int U = 4;
+        for (int i0 = begin + threadIdx.x * 8; i0 < end; i0 += U * ARGMAX_THREADS * 8) {
+            uint4 u[U];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    best = umax64(best, pack_key(w[j] & 0xffffu, i + 2 * j));
-                    best = umax64(best, pack_key(w[j] >> 16, i + 2 * j + 1));
+            for (int k = 0; k < U; ++k) {
+                const int i = i0 + k * ARGMAX_THREADS * 8;
+                u[k] = make_uint4(0u, 0u, 0u, 0u);
+                if (i + 8 <= end)
+                    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                 : "=r"(u[k].x), "=r"(u[k].y), "=r"(u[k].z), "=r"(u[k].w) : "l"(p + i));
+            }
+#pragma unroll
+            for (int k = 0; k < U; ++k) {
+                const int i = i0 + k * ARGMAX_THREADS * 8;
+                if (i + 8 <= end) {
+                    const uint32_t w[4] = {u[k].x, u[k].y, u[k].z, u[k].w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        best = umax64(best, pack_key(w[j] & 0xffffu, i + 2 * j));
+                        best = umax64(best, pack_key(w[j] >> 16, i + 2 * j + 1));
+                    }
+                } else if (i < end) {
+                    for (int j = i; j < end; ++j) best = umax64(best, pack_key(p[j], j));
                 }
-            } else {
-                for (int j = i; j < end; ++j) best = umax64(best, pack_key(p[j], j));
             }
         }
     } else {

@@ -158,6 +158,7 @@ heads_resblock_kernel(int B, int H, int K, const __nv_bfloat16 *__restrict__ hid
         float acc[NB];
 #pragma unroll
         for (int b = 0; b < NB; ++b) acc[b] = 0.f;
+#pragma unroll 4
         for (int h0 = lane * 8; h0 < H; h0 += 256) {
             float wf[8];
             bf16x8_to_float(ld_stream(w + h0), wf);
