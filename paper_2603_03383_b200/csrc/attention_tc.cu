@@ -221,8 +221,8 @@ __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
             ptx::bulk_wait_all();
             TRACE(51);   // partial left shared memory and is written
             ptx::fence_proxy_async_all();
-            __threadfence();
-            atomicAdd(p.arrive + grp, 1);
+            // release-arrive without waiting for the counter's old value
+            asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(p.arrive + grp) : "memory");
             TRACE(52);   // arrived
             const long long t0 = clock64();
             while (ld_acquire(p.arrive + grp) < nsplit)
