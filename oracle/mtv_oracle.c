@@ -20,7 +20,9 @@
  *   single-query causal attention over [prefix ; root-to-node path] computed
  *   by a library routine, closed forms for equal keys and an empty prefix;
  *   accept — brute-force sequential greedy decoding of a toy model; compaction
- *   — one-at-a-time append.  No function here is "parity unpinned".
+ *   — one-at-a-time append; LM head — one-hot hidden states that select a weight column,
+ *   a hand-computed 3x4 case, planted ties, a library matrix product.  No function here is
+ *   "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -290,4 +292,31 @@ void mtv_ref_rope(int B, int T, int Hq, int Hkv, int D,
                 }
             }
         }
+}
+
+/* ------------------------------------------------------ LM head + per-node argmax
+ * The base model's last projection as the acceptance of Section 3.2 uses it: at every tree node
+ * m the most likely token  am[m] = argmax_v z[m][v],  z[m][v] = sum_h x[m][h] W[v][h]
+ * (ties: lowest v).  x [M][H] and W [V][H] are bf16.  zmax[m] = z[m][am[m]]; z2[m] = the largest
+ * z[m][v] over v != am[m] (-inf if V == 1), which tells a test how decisive the argmax was.
+ * z_out (may be NULL) receives all logits [M][V].
+ */
+void mtv_ref_lm_head_argmax(int M, int H, int V, const uint16_t *x, const uint16_t *W,
+                            int32_t *am, double *zmax, double *z2, double *z_out)
+{
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        int best = -1;
+        double bz = 0.0, second = -INFINITY;
+        for (int v = 0; v < V; ++v) {
+            double z = 0.0;
+            for (int h = 0; h < H; ++h)
+                z += bf16_to_double(x[(size_t)m * H + h]) * bf16_to_double(W[(size_t)v * H + h]);
+            if (z_out) z_out[(size_t)m * V + v] = z;
+            if (best < 0) { best = v; bz = z; }
+            else if (z > bz) { second = bz; bz = z; best = v; }
+            else if (z > second) second = z;
+        }
+        am[m] = best; zmax[m] = bz; z2[m] = second;
+    }
 }

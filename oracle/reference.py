@@ -165,3 +165,17 @@ def rope(q, k_new, seq_lens, depth, theta=10000.0):
     lib().mtv_ref_rope(B, T, Hq, Hkv, D, _p(q), _p(k_new), _p(seq_lens), _p(depth), C.c_double(theta), _p(q_out),
                        _p(k_out))
     return q_out, k_out
+
+
+def lm_head_argmax(x, W, want_logits=False):
+    """LM head + per-node argmax: x [M,H], W [V,H] bf16 -> (am int32 [M], zmax, z2 float64 [M][, z [M,V]])."""
+    M, H = x.shape
+    V = W.shape[0]
+    assert x.dtype == W.dtype == torch.bfloat16 and W.shape[1] == H
+    x, W = x.contiguous(), W.contiguous()
+    am = torch.empty(M, dtype=torch.int32)
+    zmax = torch.empty(M, dtype=torch.float64)
+    z2 = torch.empty(M, dtype=torch.float64)
+    z = torch.empty(M, V, dtype=torch.float64) if want_logits else None
+    lib().mtv_ref_lm_head_argmax(M, H, V, _p(x), _p(W), _p(am), _p(zmax), _p(z2), _p(z))
+    return (am, zmax, z2, z) if want_logits else (am, zmax, z2)
