@@ -185,6 +185,33 @@ int tree_accept(const mtv_tree_t *tree, int B, int V, const mtv_bf16 *logits, co
                 int32_t *next_root, void *ws, size_t ws_bytes, void *stream);
 
 /* ---------------------------------------------------------------------------
+ * LM-head projection fused with the per-node argmax — the base model's last layer as the
+ * acceptance of Section 3.2 consumes it: only the most likely token at every tree node is
+ * needed, so the [B][T][V] logits are never written.
+ *   am[b][i]     = argmax_v <x[b][i], W[v]>                      (ties: lowest v)
+ *   am_val[b][i] = that maximum
+ * bf16 inputs, products accumulated in fp32 on the tensor cores; the comparison is made on
+ * the fp32 sums (no rounding to bf16 first, unlike tree_accept on stored bf16 logits).
+ * All pointers device.  x [B][T][H] (final hidden state of the tree nodes, after the last
+ * norm), W [V][H] row-major (the LM head), both bf16, 16-byte aligned; H a multiple of 64.
+ * keys [B*T] uint64, written by the call (zeroed, then filled): per node the order-preserving
+ * image of the maximum in the high word and 0xffffffff - argmax in the low word — the input of
+ * tree_accept_keys.  am [B*T] int32 and am_val [B*T] float may be NULL (am_val only if am is).
+ * No workspace.  A wait inside the kernel that runs out sets the tree's device error word
+ * (mtv_device_error) to MTV_ERR_TIMEOUT; the outputs are then undefined.
+ * Errors: MTV_ERR_INVALID_ARG (null / misaligned pointers, sizes < 1),
+ * MTV_ERR_UNSUPPORTED_SHAPE (H), MTV_ERR_CUDA.
+ */
+int lm_head_argmax(const mtv_tree_t *tree, int B, int H, int V, const mtv_bf16 *x, const mtv_bf16 *W,
+                   int32_t *am, float *am_val, unsigned long long *keys, void *stream);
+
+/* tree_accept on the keys of lm_head_argmax instead of stored logits: same outputs, same
+ * acceptance rule (Section 3.2), am[b][i] taken from keys[b*T + i].  All pointers device. */
+int tree_accept_keys(const mtv_tree_t *tree, int B, const unsigned long long *keys, const int32_t *tree_tok,
+                     int32_t *accept_len, int32_t *best_path, int32_t *acc_nodes, int32_t *acc_tok,
+                     int32_t *next_root, void *stream);
+
+/* ---------------------------------------------------------------------------
  * tree_accept without a workspace — the paper has no counterpart; this is a convenience of
  * the library.  Same inputs, outputs and results as tree_accept, but the scratch (the
  * per-chunk argmax keys) sits in a 64 KB array that is part of the library image, so the call

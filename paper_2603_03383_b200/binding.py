@@ -26,7 +26,8 @@ EXPORTS = ["tree_build_static", "tree_gen_cartesian", "tree_gen_rank_prior", "tr
            "mtv_workspace_bytes", "medusa_heads_topk", "tree_verify_attention", "tree_accept",
            "kv_compact_accepted", "mtv_verify_step", "mtv_verify_step_host", "mtv_last_error",
            "mtv_set_kernel_taps", "mtv_kernel_taps_used", "mtv_device_error",
-           "tree_accept_static_scratch", "tree_accept_static_scratch_capacity", "tree_kv_append_rope"]
+           "tree_accept_static_scratch", "tree_accept_static_scratch_capacity", "tree_kv_append_rope",
+           "lm_head_argmax", "tree_accept_keys"]
 
 
 class MtvError(RuntimeError):
@@ -100,6 +101,8 @@ def lib():
         L.tree_accept_static_scratch_capacity.restype = sz
         L.tree_kv_append_rope.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, i64, i64, i64, i32, vp, C.c_float,
                                           vp, vp]
+        L.lm_head_argmax.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+        L.tree_accept_keys.argtypes = [vp, i32] + [vp] * 7 + [vp]
         _lib = L
     return _lib
 
@@ -229,6 +232,19 @@ def tree_accept(tree, logits, tree_tok, accept_len, best_path, acc_nodes, acc_to
     _check(lib().tree_accept(tree.handle, B, V, _ptr(logits), _ptr(tree_tok), _ptr(accept_len), _ptr(best_path),
                              _ptr(acc_nodes), _ptr(acc_tok), _ptr(next_root), p, n, _stream(stream)),
            "tree_accept")
+
+
+def lm_head_argmax(tree, x, W, keys, am=None, am_val=None, stream=None):
+    """x [B][T][H], W [V][H] bf16; keys [B*T] int64 storage for the uint64 keys (see include/mtv.h)."""
+    B, T, H = x.shape
+    _check(lib().lm_head_argmax(tree.handle, B, H, W.shape[0], _ptr(x), _ptr(W),
+                                _ptr(am), _ptr(am_val), _ptr(keys), _stream(stream)), "lm_head_argmax")
+
+
+def tree_accept_keys(tree, B, keys, tree_tok, accept_len, best_path, acc_nodes, acc_tok, next_root, stream=None):
+    _check(lib().tree_accept_keys(tree.handle, B, _ptr(keys), _ptr(tree_tok), _ptr(accept_len), _ptr(best_path),
+                                  _ptr(acc_nodes), _ptr(acc_tok), _ptr(next_root), _stream(stream)),
+           "tree_accept_keys")
 
 
 def tree_accept_static_scratch(tree, logits, tree_tok, accept_len, best_path, acc_nodes, acc_tok, next_root,

@@ -155,6 +155,23 @@ extern "C" int tree_accept(const mtv_tree_t *tree, int B, int V, const mtv_bf16 
     return MTV_OK;
 }
 
+// Acceptance from per-node argmax keys (what lm_head_argmax leaves): the finish kernel alone, with
+// one key per node.
+extern "C" int tree_accept_keys(const mtv_tree_t *tree, int B, const unsigned long long *keys, const int32_t *tree_tok,
+                                int32_t *accept_len, int32_t *best_path, int32_t *acc_nodes, int32_t *acc_tok,
+                                int32_t *next_root, void *stream) {
+    using namespace mtv;
+    if (!tree || !tree->on_device || !keys || !tree_tok || !accept_len || !best_path || !acc_nodes || !acc_tok ||
+        !next_root || B < 1)
+        return MTV_ERR_INVALID_ARG;
+    if (tree->P > 255) return MTV_ERR_UNSUPPORTED_SHAPE;
+    accept_finish_kernel<<<B, 128, 0, (cudaStream_t)stream>>>(tree->T, tree->K, tree->P, 1, keys, tree_tok,
+                                                              tree->d_retrieve, accept_len, best_path, acc_nodes,
+                                                              acc_tok, next_root);
+    MTV_CUDA_CHECK(cudaGetLastError());
+    return MTV_OK;
+}
+
 // ---------------------------------------------------------------------------
 // tree_accept for callers that must not allocate device memory (the paper has no counterpart).
 // Its scratch — the per-chunk argmax keys that tree_accept keeps in the caller's workspace —
