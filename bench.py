@@ -58,8 +58,9 @@ def peaks():
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
 # profiles/, keyed by tap name, with the hash of the kernel's source at capture time: a changed kernel reports null.
 NCU_TRAFFIC = {
-    "attn_partial": ("attention_tc.cu", "5bb0db1477ad2184", 34.415e6 + 0.01e6),
-    "heads_vocab_topk": ("heads.cu", "be18a2d50043db27", 4.2951e9 + 4.5e6),
+    "attn_partial": ("attention_tc.cu", "972d0fab6bdae3e0", 34.415e6 + 0.013e6),
+    "heads_vocab_topk": ("heads.cu", "080f8e7cc04e0d45", 4.2951e9 + 4.5e6),
+    "lm_head_argmax": ("lm_head.cu", "bb9bd39d12c92842", 1.0759e9 + 3.8e6),
 }
 
 
@@ -314,6 +315,7 @@ def run_ours(args):
         return
     pk = peaks()
     alg = algorithmic_bytes(w, tree, n_layers, P["lens"].tolist())
+    lm = time_lm_head(tree, w, P, dev)
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W_steps,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -363,6 +365,12 @@ def run_ours(args):
                                 "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": ach / pk["hbm_gbs"],
                                 "frac_of_8tbs": ach / 8000.0, "avg_call_us": a_ms * 1e3,
                                 "algorithmic_bytes_per_launch": alg["attn_per_layer"]}
+    lm_bytes = w.V * w.H * 2 + 2 * w.B * tree.T * w.H
+    out["beyond_the_step"] = {"lm_head_argmax": {
+        "what": "LM head with fused per-node argmax + acceptance from its keys (not part of the timed step)",
+        "us_per_call": lm * 1e3, "algorithmic_bytes": lm_bytes, "achieved_gbs": lm_bytes / lm / 1e6,
+        "frac_of_measured_hbm": lm_bytes / lm / 1e6 / pk["hbm_gbs"],
+        "tflops": 2.0 * w.B * tree.T * w.V * w.H / lm / 1e9}}
     if not args.no_cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(w, P, n_layers, budget_s=25.0)
     elif not args.no_cpu_baseline:
@@ -370,6 +378,32 @@ def run_ours(args):
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def time_lm_head(tree, w, P, dev, iters=20):
+    """ms per call of lm_head_argmax + tree_accept_keys on the workload's B, T, H, V (the first Medusa head's
+    vocabulary matrix stands in for the LM head: same shape, same distribution), back-to-back launches."""
+    import torch
+    from paper_2603_03383_b200 import binding, synth
+    B, T, K = w.B, tree.T, w.K
+    x = synth.normal_bf16(w.seed, 77, (B, T, w.H), device=dev)
+    W = P["W2"][0]
+    keys = torch.zeros(B * T, dtype=torch.int64, device=dev)
+    i32 = lambda *s: torch.zeros(*s, dtype=torch.int32, device=dev)
+    outs = [i32(B), i32(B), i32(B, K + 1), i32(B, K + 1), i32(B)]
+    def call():
+        binding.lm_head_argmax(tree, x, W, keys)
+        binding.tree_accept_keys(tree, B, keys, P["tree_tok"], *outs)
+    for _ in range(3):
+        call()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(iters):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
 
 
 def _sample_plan(w, T, n_layers, est_full_s, budget_s):

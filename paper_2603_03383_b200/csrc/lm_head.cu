@@ -7,8 +7,10 @@
 // arithmetic intensity is M flop per weight byte, so HBM bounds it; the vocabulary rows are the
 // MMA's M dimension, the nodes its N dimension:
 //   D[128 vocabulary rows][N nodes] += W_tile[128][64 k] . X[N][64 k]^T      (both operands K-major)
-// One persistent CTA per SM walks pairs of vocabulary tiles (256 rows), so that a chunk of X fetched
-// from L2 serves two weight tiles.  Warp roles: TMA producer (ring of stages, one stage = 64
+// One persistent CTA per SM walks pairs of vocabulary tiles, so that a chunk of X fetched from L2
+// serves two weight tiles.  A tile holds R <= 128 rows, R chosen by the host so that every CTA gets
+// the same number of pairs (V = 32000 on 148 SMs: 112 rows); the MMA spans 128 rows all the same and
+// the rows past R, whatever the shared memory held, are left out of the maximum.  Warp roles: TMA producer (ring of stages, one stage = 64
 // columns of 256 weight rows and of the N node rows), MMA issuer (accumulators in tensor memory,
 // double-buffered: the epilogue of one pair overlaps the MMAs of the next), four epilogue warps
 // (one thread per vocabulary row: order-preserving (value, ~index) keys, butterfly max over the
@@ -32,6 +34,9 @@ struct LmParams {
     unsigned long long *keys;   // [M] best (value, ~index) per node, zero before the launch
     int32_t *dev_error;
     int M, H, V, N;             // N = nodes per pass (64 or 128)
+    int R;                      // vocabulary rows per tile (<= 128, a multiple of 8), chosen so that the tiles
+                                // divide evenly among the CTAs; the MMA still spans 128 rows, the rest is ignored
+    int n_pairs;                // tile pairs over the vocabulary
     int n_stages;
     uint32_t stage_bytes;
 };
@@ -122,7 +127,7 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_co
     // passes are neighbours in launch order, so all but the first find those rows in L2
     const int pass = blockIdx.x;                         // nodes [pass N, pass N + N)
     const int cta = blockIdx.y, n_cta = gridDim.y;
-    const int n_pairs = (p.V + 255) / 256;
+    const int n_pairs = p.n_pairs, R = p.R;
     const int my_pairs = cta < n_pairs ? (n_pairs - cta + n_cta - 1) / n_cta : 0;
     const int n_kc = p.H / LM_KC;
     const uint32_t x_off = LM_W_BYTES;                   // X chunk sits after the weight chunk in a stage
@@ -131,15 +136,15 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_co
         // ---------------------------------------------------------------- TMA producer
         int it = 0;
         for (int q = 0; q < my_pairs && !*abort_flag; ++q) {
-            const int row0 = (cta + q * n_cta) * 256;
+            const int row0 = (cta + q * n_cta) * 2 * R;
             for (int kc = 0; kc < n_kc; ++kc, ++it) {
                 const int s = it % NST, use = it / NST;
                 if (use > 0 && !ptx::mbar_wait(empty(s), (use - 1) & 1)) { *abort_flag = 1; break; }
                 if (lane == 0) {
                     const uint32_t base = ring + s * p.stage_bytes;
-                    ptx::mbar_arrive_expect_tx(full(s), LM_W_BYTES + N * 128);
+                    ptx::mbar_arrive_expect_tx(full(s), (uint32_t)(2 * R + N) * 128u);
                     tma_load_2d(base, &w_map, full(s), kc * LM_KC, row0);                 // rows past V arrive as zeros
-                    tma_load_2d(base + LM_W_BYTES / 2, &w_map, full(s), kc * LM_KC, row0 + 128);
+                    tma_load_2d(base + LM_W_BYTES / 2, &w_map, full(s), kc * LM_KC, row0 + R);
                     tma_load_2d(base + x_off, &x_map, full(s), kc * LM_KC, pass * N);      // rows past M arrive as zeros
                 }
                 __syncwarp();
@@ -185,10 +190,11 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_co
             if (ok) ok = ptx::mbar_wait(acc_full(u), (q >> 1) & 1);
             __syncwarp();
             ptx::tc_fence_after();
-            const int row0 = (cta + q * n_cta) * 256;
+            const int row0 = (cta + q * n_cta) * 2 * R;
 #pragma unroll 1
             for (int t = 0; t < 2; ++t) {
-                const int v = row0 + t * 128 + warp * 32 + lane;       // this thread's vocabulary row
+                const int r = warp * 32 + lane;
+                const int v = r < R ? row0 + t * R + r : p.V;          // this thread's vocabulary row (none past R)
 #pragma unroll 1
                 for (int c = 0; c < N / 32; ++c) {
                     uint32_t acc[32];
@@ -287,7 +293,6 @@ extern "C" int lm_head_argmax(const mtv_tree_t *tree, int B, int H, int V, const
     const int passes = (M + N - 1) / N;
         cudaStream_t st = (cudaStream_t)stream;
     CUtensorMap w_map, x_map;
-    if (!lm_map(&w_map, W, V, H, 128) || !lm_map(&x_map, x, M, H, N)) return MTV_ERR_CUDA;
     LmParams p;
     p.keys = keys; p.dev_error = tree->d_error; p.M = M; p.H = H; p.V = V; p.N = N;
     p.stage_bytes = LM_W_BYTES + N * 128;
@@ -302,9 +307,14 @@ extern "C" int lm_head_argmax(const mtv_tree_t *tree, int B, int H, int V, const
     }
     MTV_CUDA_CHECK(cudaMemsetAsync(keys, 0, (size_t)M * 8, st));
     int ctas = sm_count() / passes;                      // per pass; one CTA per SM in all
-    const int n_pairs = (V + 255) / 256;
-    if (ctas > n_pairs) ctas = n_pairs;
+    const int min_pairs = (V + 255) / 256;
+    if (ctas > (V + 63) / 64) ctas = (V + 63) / 64;      // no tile below 32 rows
     if (ctas < 1) ctas = 1;
+    // every CTA walks the same number of tile pairs; the tile height shrinks until they just cover V
+    const int rounds = (min_pairs + ctas - 1) / ctas;
+    p.n_pairs = ctas * rounds;
+    p.R = ((V + 2 * p.n_pairs - 1) / (2 * p.n_pairs) + 7) / 8 * 8;
+    if (!lm_map(&w_map, W, V, H, p.R) || !lm_map(&x_map, x, M, H, N)) return MTV_ERR_CUDA;
     const dim3 grid(passes, ctas);
     if (N == 64) lm_head_argmax_kernel<64><<<grid, LM_THREADS, smem, st>>>(w_map, x_map, p);
     else lm_head_argmax_kernel<128><<<grid, LM_THREADS, smem, st>>>(w_map, x_map, p);
