@@ -275,6 +275,12 @@ typedef struct {
     int32_t *accept_len, *best_path, *acc_nodes, *acc_tok, *next_root;
     int32_t *status;           /* [B] or NULL */
     void *ws; size_t ws_bytes;
+    /* Optional: the acceptance takes the base model's argmax from the fused LM head instead of
+     * stored logits.  If x_final ([B][T][H], final hidden state of the tree nodes) and W_lm
+     * ([V][H]) are both non-NULL, the step runs lm_head_argmax on them followed by
+     * tree_accept_keys and never reads `logits` (which may then be NULL); the keys live at the
+     * start of ws.  The host variant uploads x_final instead of logits. */
+    const mtv_bf16 *x_final, *W_lm;
 } mtv_step_args;
 
 int mtv_verify_step(const mtv_tree_t *tree, const mtv_step_args *args, void *stream);

@@ -63,7 +63,8 @@ class StepArgs(C.Structure):
                 ("out_layers", C.c_void_p),
                 ("accept_len", C.c_void_p), ("best_path", C.c_void_p), ("acc_nodes", C.c_void_p),
                 ("acc_tok", C.c_void_p), ("next_root", C.c_void_p), ("status", C.c_void_p),
-                ("ws", C.c_void_p), ("ws_bytes", C.c_size_t)]
+                ("ws", C.c_void_p), ("ws_bytes", C.c_size_t),
+                ("x_final", C.c_void_p), ("W_lm", C.c_void_p)]
 
 
 _lib = None

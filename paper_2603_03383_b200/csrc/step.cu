@@ -14,6 +14,21 @@ extern "C" size_t mtv_workspace_bytes(const mtv_tree_t *tree, int B, int H, int 
     return need;
 }
 
+// Acceptance of a step: from stored logits, or from the fused LM head when the caller gave its operands
+// (the per-node keys then sit at the start of the workspace, which no other kernel uses at that point).
+static int step_accept(const mtv_tree_t *tree, const mtv_step_args *a, void *stream) {
+    if (a->x_final && a->W_lm) {
+        if (!a->ws || a->ws_bytes < (size_t)a->B * tree->T * sizeof(unsigned long long)) return MTV_ERR_WORKSPACE;
+        unsigned long long *keys = static_cast<unsigned long long *>(a->ws);
+        const int rc = lm_head_argmax(tree, a->B, a->H, a->V, a->x_final, a->W_lm, nullptr, nullptr, keys, stream);
+        if (rc != MTV_OK) return rc;
+        return tree_accept_keys(tree, a->B, keys, a->tree_tok, a->accept_len, a->best_path, a->acc_nodes, a->acc_tok,
+                                a->next_root, stream);
+    }
+    return tree_accept(tree, a->B, a->V, a->logits, a->tree_tok, a->accept_len, a->best_path, a->acc_nodes, a->acc_tok,
+                       a->next_root, a->ws, a->ws_bytes, stream);
+}
+
 extern "C" int mtv_verify_step(const mtv_tree_t *tree, const mtv_step_args *a, void *stream) {
     if (!tree || !a || !a->k_caches_host || !a->v_caches_host) return MTV_ERR_INVALID_ARG;
     int rc = medusa_heads_topk(tree, a->B, a->H, a->V, a->hidden, a->W1, a->b1, a->W2, a->root_tok, a->cand,
@@ -26,8 +41,7 @@ extern "C" int mtv_verify_step(const mtv_tree_t *tree, const mtv_step_args *a, v
                                    a->scale, a->out_layers + l * per_layer, a->status, a->ws, a->ws_bytes, stream);
         if (rc != MTV_OK) return rc;
     }
-    rc = tree_accept(tree, a->B, a->V, a->logits, a->tree_tok, a->accept_len, a->best_path, a->acc_nodes, a->acc_tok,
-                     a->next_root, a->ws, a->ws_bytes, stream);
+    rc = step_accept(tree, a, stream);
     if (rc != MTV_OK) return rc;
     return kv_compact_accepted(tree, a->B, a->Hkv, a->D, a->n_layers, a->k_caches, a->v_caches, a->stride_b,
                                a->stride_h, a->stride_t, a->Lcap, a->seq_lens, a->accept_len, a->acc_nodes, a->status,
@@ -75,7 +89,10 @@ extern "C" int mtv_verify_step_host(const mtv_tree_t *tree, const mtv_step_args 
     MTV_CUDA_CHECK(cudaMemcpyAsync((void *)d->root_tok, h->root_tok, B * 4, cudaMemcpyHostToDevice, st));
     MTV_CUDA_CHECK(cudaMemcpyAsync((void *)d->q_layers, h->q_layers, q_bytes, cudaMemcpyHostToDevice, up));
     MTV_CUDA_CHECK(cudaEventRecord(g_aux.q_up, up));
-    MTV_CUDA_CHECK(cudaMemcpyAsync((void *)d->logits, h->logits, B * T * d->V * 2, cudaMemcpyHostToDevice, up));
+    if (d->x_final && d->W_lm)
+        MTV_CUDA_CHECK(cudaMemcpyAsync((void *)d->x_final, h->x_final, B * T * d->H * 2, cudaMemcpyHostToDevice, up));
+    else
+        MTV_CUDA_CHECK(cudaMemcpyAsync((void *)d->logits, h->logits, B * T * d->V * 2, cudaMemcpyHostToDevice, up));
     MTV_CUDA_CHECK(cudaEventRecord(g_aux.logits_up, up));
     // heads
     int rc = medusa_heads_topk(tree, d->B, d->H, d->V, d->hidden, d->W1, d->b1, d->W2, d->root_tok, d->cand, d->cand_logit,
@@ -102,8 +119,7 @@ extern "C" int mtv_verify_step_host(const mtv_tree_t *tree, const mtv_step_args 
     }
     // acceptance and compaction
     MTV_CUDA_CHECK(cudaStreamWaitEvent(st, g_aux.logits_up, 0));
-    rc = tree_accept(tree, d->B, d->V, d->logits, d->tree_tok, d->accept_len, d->best_path, d->acc_nodes, d->acc_tok,
-                     d->next_root, d->ws, d->ws_bytes, stream);
+    rc = step_accept(tree, d, stream);
     if (rc != MTV_OK) return rc;
     rc = kv_compact_accepted(tree, d->B, d->Hkv, d->D, d->n_layers, d->k_caches, d->v_caches, d->stride_b, d->stride_h,
                              d->stride_t, d->Lcap, d->seq_lens, d->accept_len, d->acc_nodes, d->status, stream);

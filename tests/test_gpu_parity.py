@@ -247,7 +247,7 @@ def test_kv_compaction(D, n_layers, B, Hkv):
 
 
 # -------------------------------------------------------------- full step
-def _step_case(B, H, V, Hq, Hkv, D, n_layers, kind, K, topk, T, lens, seed, host=False):
+def _step_case(B, H, V, Hq, Hkv, D, n_layers, kind, K, topk, T, lens, seed, host=False, lm_head=False):
     tb, tree = make_tree(kind, K, topk, T)
     T = tree.T
     Lcap = max(lens) + T
@@ -255,6 +255,15 @@ def _step_case(B, H, V, Hq, Hkv, D, n_layers, kind, K, topk, T, lens, seed, host
     logits, planted = synth.planted_logits(B, T, V, K, tt_ref, tb["parent"], tb["rank"], seed, p_accept=(0.6, 0.9))
     acc_ref = ref.tree_accept(ref.node_argmax(logits), tt_ref, tb)
     assert torch.equal(acc_ref["accept_len"], planted)
+    if lm_head:
+        # the same planted next tokens, this time as the argmax of an LM head: the hidden state of node i is
+        # the weight row of its token plus noise; the step gets (x_final, W_lm) and no logits
+        target = ref.node_argmax(logits).long()
+        W_lm = synth.normal_bf16(seed, 901, (V, H))
+        x_final = (W_lm[target.flatten()].float().reshape(B, T, H) +
+                   0.3 * synth.normal_bf16(seed, 902, (B, T, H)).float()).to(torch.bfloat16)
+        am, zmax, z2 = ref.lm_head_argmax(x_final.reshape(B * T, H), W_lm)
+        assert torch.equal(am.long(), target.flatten()) and ((zmax - z2) > 1e-3 * zmax.abs().max()).all()
     sl = torch.tensor(lens, dtype=torch.int32)
     layers = [synth.attention_inputs(B, T, Hq, Hkv, D, Lcap, seed, layer=l) for l in range(n_layers)]
     out_ref = torch.stack([ref.tree_attention(q, k, v, sl, tb["mask"]) for q, k, v in layers])
@@ -273,17 +282,23 @@ def _step_case(B, H, V, Hq, Hkv, D, n_layers, kind, K, topk, T, lens, seed, host
                accept_len=_i32(B), best_path=_i32(B), acc_nodes=_i32(B, K + 1), acc_tok=_i32(B, K + 1),
                next_root=_i32(B), status=_i32(B), k_caches=kp, v_caches=vp, k_caches_host=kph, v_caches_host=vph,
                ws=workspace(tree, B, H, V, Hq, Hkv, D, Lcap))
+    up = ["hidden", "root_tok", "q_layers", "logits"]
+    src = dict(hidden=hidden, root_tok=root, q_layers=q_all, logits=logits)
+    if lm_head:
+        del dev["logits"]                                          # never read on this path
+        dev["x_final"], dev["W_lm"] = x_final.to(DEV), W_lm.to(DEV)
+        up[3], src["x_final"] = "x_final", x_final
+        del src["logits"]
     for name, t in dev.items():
         setattr(a, name, t.data_ptr())
     a.ws_bytes = dev["ws"].numel()
     if host:
         hb = binding.StepArgs()
-        names = ["hidden", "root_tok", "q_layers", "logits", "tree_tok", "out_layers", "accept_len", "best_path",
-                 "acc_nodes", "acc_tok", "next_root", "seq_lens"]
-        src = dict(hidden=hidden, root_tok=root, q_layers=q_all, logits=logits)
+        names = up + ["tree_tok", "out_layers", "accept_len", "best_path", "acc_nodes", "acc_tok", "next_root",
+                      "seq_lens"]
         hostbuf = {n: (src[n].clone() if n in src else torch.empty_like(dev[n], device="cpu")).pin_memory()
                    for n in names}
-        for n in ("hidden", "root_tok", "q_layers", "logits"):     # the device copies start out wrong
+        for n in up:                                               # the device copies start out wrong
             dev[n].zero_()
         for n, t in hostbuf.items():
             setattr(hb, n, t.data_ptr())
@@ -321,6 +336,14 @@ def test_full_step_batched_ragged():
 
 def test_full_step_from_host_buffers():
     _step_case(2, 256, 2000, 8, 2, 64, 2, "cartesian", 3, (4, 2, 2), 0, [90, 33], seed=8, host=True)
+
+
+def test_full_step_with_fused_lm_head():
+    _step_case(5, 256, 3000, 8, 2, 128, 2, "rank_prior", 4, (), 64, [300, 17, 0, 129, 64], seed=31, lm_head=True)
+
+
+def test_full_step_with_fused_lm_head_from_host_buffers():
+    _step_case(2, 256, 2000, 8, 2, 64, 2, "cartesian", 3, (4, 2, 2), 0, [90, 33], seed=8, host=True, lm_head=True)
 
 
 def test_generator_is_identical_on_cpu_and_gpu():
