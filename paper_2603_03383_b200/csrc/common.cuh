@@ -48,10 +48,16 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 
 // Workspace carving shared by the entry points (all offsets 256-byte aligned).
 struct HeadsWs {
-    size_t hprime_off, part_val_off, part_idx_off, counters_off, total;
+    size_t hprime_off, part_val_off, part_idx_off, counters_off, xsplit_off, total;
     int ctas_per_head, n_counters;
+    bool use_tc;   // several batch rows: vocabulary projection on the tcgen05 tensor cores
 };
 HeadsWs heads_ws_layout(const mtv_tree *t, int B, int H, int V);
+bool heads_tc_eligible(int B, int H);
+size_t heads_tc_xsplit_bytes(int K, int H);
+int launch_heads_vocab_tc(const mtv_tree *t, int B, int H, int V, const __nv_bfloat16 *W2, const int32_t *root_tok,
+                          int32_t *cand, float *cand_logit, int32_t *tree_tok, const HeadsWs &L, char *ws,
+                          cudaStream_t st);
 
 struct AttnWs {
     size_t o_off, ml_off, total;

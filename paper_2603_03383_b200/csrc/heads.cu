@@ -7,6 +7,7 @@
 // with many loads in flight; activations stay in shared memory in fp32 so that no
 // intermediate is rounded.
 #include "common.cuh"
+#include "heads_common.cuh"
 #include "sm100_ptx.cuh"
 
 namespace mtv {
@@ -77,6 +78,9 @@ HeadsWs heads_ws_layout(const mtv_tree *t, int B, int H, int V) {
     w.part_idx_off = off; off = align_up(off + (size_t)t->K * B * per_head * MTV_MAX_TOPK * sizeof(int32_t), 256);
     w.counters_off = off; off = align_up(off + (size_t)(t->K + 1) * btiles * sizeof(int32_t), 256);
     w.n_counters = (t->K + 1) * btiles;
+    w.use_tc = heads_tc_eligible(B, H);
+    w.xsplit_off = off;
+    if (w.use_tc) off = align_up(off + heads_tc_xsplit_bytes(t->K, H), 256);
     w.total = off;
     return w;
 }
@@ -126,11 +130,6 @@ __device__ __forceinline__ void warp_sum_scatter(float (&v)[N], int lane) {
             v[0] += __shfl_xor_sync(0xffffffffu, v[0], bit);
         }
     }
-}
-
-// (value, id) ordering of the candidate lists: larger value first, equal values by smaller id.
-__device__ __forceinline__ bool cand_before(float va, int ia, float vb, int ib) {
-    return va > vb || (va == vb && ia < ib);
 }
 
 // ---------------------------------------------------------------------------
@@ -199,22 +198,6 @@ heads_resblock_kernel(int B, int H, int K, const __nv_bfloat16 *__restrict__ hid
 // when it beats the list's last entry.  Afterwards the warps' lists are merged per CTA;
 // the last CTA of a head (atomic ticket, no waiting) merges the CTAs' lists into the
 // candidate buffer, and the last head to finish expands the candidates into tree tokens.
-struct VocabParams {
-    int B, H, V, K, T, C;
-    const __nv_bfloat16 *W2;
-    const float *hprime;
-    const int32_t *kd_arr, *off_arr, *tree_indices, *root_tok;
-    float *part_val;
-    int32_t *part_idx;
-    int32_t *counters;   // [btiles][K + 1], zeroed by the residual-block kernel
-    int32_t *cand;
-    float *cand_logit;
-    int32_t *tree_tok;
-    int32_t *dev_error;
-    int rows_per_stage, n_stages, n_it;
-    uint32_t stage_bytes, xs_off, lists_off, zbuf_off, bars_off;
-};
-
 template <int NB>
 __global__ void __launch_bounds__(VT_THREADS, 1)
 heads_vocab_topk_kernel(const VocabParams p) {
@@ -223,7 +206,6 @@ heads_vocab_topk_kernel(const VocabParams p) {
     float *lval = reinterpret_cast<float *>(smem + p.lists_off);          // [CONS_WARPS][NB][16]
     int32_t *lidx = reinterpret_cast<int32_t *>(lval + VT_CONS_WARPS * NB * MTV_MAX_TOPK);
     const uint32_t bars = ptx::smem_u32(smem + p.bars_off);               // full[n_stages], empty[n_stages]
-    __shared__ int s_flag;
     __shared__ int s_abort;
 
     const int k = blockIdx.y, bz = blockIdx.z, b0 = bz * NB;
@@ -454,76 +436,7 @@ heads_vocab_topk_kernel(const VocabParams p) {
         return;
     }
 
-    // ---- merge the warps' lists: rank each entry among all CONS_WARPS*kd entries of its batch row
-    for (int e = threadIdx.x; e < NB * VT_CONS_WARPS * MTV_MAX_TOPK; e += VT_THREADS) {
-        const int b = e / (VT_CONS_WARPS * MTV_MAX_TOPK);
-        const int w = (e / MTV_MAX_TOPK) % VT_CONS_WARPS, sl = e % MTV_MAX_TOPK;
-        if (sl >= kd || b0 + b >= p.B) continue;
-        const float zz = lval[(w * NB + b) * MTV_MAX_TOPK + sl];
-        const int id = lidx[(w * NB + b) * MTV_MAX_TOPK + sl];
-        int rank = 0;
-        for (int w2 = 0; w2 < VT_CONS_WARPS; ++w2)
-            for (int s2 = 0; s2 < kd; ++s2) {
-                const float z2 = lval[(w2 * NB + b) * MTV_MAX_TOPK + s2];
-                const int id2 = lidx[(w2 * NB + b) * MTV_MAX_TOPK + s2];
-                // unused slots all carry the same sentinel: order them by position
-                if (cand_before(z2, id2, zz, id) || (z2 == zz && id2 == id && (w2 * MTV_MAX_TOPK + s2) < (w * MTV_MAX_TOPK + sl)))
-                    ++rank;
-            }
-        if (rank < kd) {
-            const size_t o = (((size_t)k * p.B + b0 + b) * per + blockIdx.x) * MTV_MAX_TOPK + rank;
-            p.part_val[o] = zz;
-            p.part_idx[o] = id;
-        }
-    }
-    // ---- last CTA of this head merges the CTAs' lists (ticket: nobody waits)
-    int32_t *counters = p.counters + (size_t)bz * (p.K + 1);
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) s_flag = atomicAdd(&counters[k], 1) == per - 1;
-    __syncthreads();
-    if (!s_flag) return;
-    __threadfence();
-    {
-        float *mval = reinterpret_cast<float *>(smem);                     // the ring is idle now
-        int32_t *midx = reinterpret_cast<int32_t *>(mval + per * MTV_MAX_TOPK);
-        const int n = per * kd, off = p.off_arr[k];
-        for (int b = 0; b < NB && b0 + b < p.B; ++b) {
-            __syncthreads();
-            for (int e = threadIdx.x; e < n; e += VT_THREADS) {
-                const size_t o = (((size_t)k * p.B + b0 + b) * per + e / kd) * MTV_MAX_TOPK + e % kd;
-                mval[e] = __ldcg(p.part_val + o);
-                midx[e] = __ldcg(p.part_idx + o);
-            }
-            __syncthreads();
-            for (int e = threadIdx.x; e < n; e += VT_THREADS) {
-                const float zz = mval[e];
-                const int id = midx[e];
-                int rank = 0;
-                for (int e2 = 0; e2 < n && rank < kd; ++e2)
-                    if (cand_before(mval[e2], midx[e2], zz, id) || (mval[e2] == zz && midx[e2] == id && e2 < e)) ++rank;
-                if (rank < kd) {
-                    p.cand[(size_t)(b0 + b) * p.C + off + rank] = id;
-                    if (p.cand_logit) p.cand_logit[(size_t)(b0 + b) * (p.C - 1) + off - 1 + rank] = zz;
-                }
-            }
-        }
-    }
-    // ---- last head of this batch tile expands the candidates into the tree tokens
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) s_flag = atomicAdd(&counters[p.K], 1) == p.K - 1;
-    __syncthreads();
-    if (!s_flag) return;
-    __threadfence();
-    for (int e = threadIdx.x; e < NB * p.T; e += VT_THREADS) {
-        const int b = b0 + e / p.T, i = e % p.T;
-        if (b >= p.B) break;
-        const int slot = p.tree_indices[i];
-        const int32_t root = p.root_tok[b];
-        if (i == 0) p.cand[(size_t)b * p.C] = root;
-        p.tree_tok[(size_t)b * p.T + i] = slot == 0 ? root : __ldcg(p.cand + (size_t)b * p.C + slot);
-    }
+    vocab_tail(p, NB, VT_CONS_WARPS, lval, lidx, smem, k, bz, b0, per, kd, p.xs_off);
 }
 
 template <int NB>
@@ -535,8 +448,11 @@ static int launch_heads(const mtv_tree *t, int B, int H, int V, const __nv_bfloa
     const int btiles = (B + NB - 1) / NB;
     const size_t sm1 = (size_t)NB * H * sizeof(float);
     const VocabSmem S = vocab_smem_plan(NB, H, L.ctas_per_head);
-    if (sm1 > VT_SMEM_MAX || S.total == 0) return MTV_ERR_UNSUPPORTED_SHAPE;
-    if (NB > 1 && S.rows_per_stage < (NB >= 4 ? 4 : 2)) return MTV_ERR_UNSUPPORTED_SHAPE;   // rows too long for a block of rows per stage
+    if (sm1 > VT_SMEM_MAX) return MTV_ERR_UNSUPPORTED_SHAPE;
+    if (!L.use_tc) {
+        if (S.total == 0) return MTV_ERR_UNSUPPORTED_SHAPE;
+        if (NB > 1 && S.rows_per_stage < (NB >= 4 ? 4 : 2)) return MTV_ERR_UNSUPPORTED_SHAPE;   // rows too long for a block of rows per stage
+    }
     static bool attr_done = false;
     if (!attr_done) {
         MTV_CUDA_CHECK(cudaFuncSetAttribute(heads_resblock_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, VT_SMEM_MAX));
@@ -552,6 +468,7 @@ static int launch_heads(const mtv_tree *t, int B, int H, int V, const __nv_bfloa
         heads_resblock_kernel<NB><<<dim3(g1, btiles), HEADS_THREADS, sm1, st>>>(B, H, t->K, hidden, W1, b1, hprime,
                                                                                counters, L.n_counters);
     }
+    if (L.use_tc) return launch_heads_vocab_tc(t, B, H, V, W2, root_tok, cand, cand_logit, tree_tok, L, ws, st);
     VocabParams p;
     p.B = B; p.H = H; p.V = V; p.K = t->K; p.T = t->T; p.C = t->C;
     p.W2 = W2; p.hprime = hprime;

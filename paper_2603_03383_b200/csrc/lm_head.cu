@@ -19,6 +19,7 @@
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
+#include "tma_host.cuh"
 
 namespace mtv {
 
@@ -253,33 +254,6 @@ __global__ void lm_head_finish_kernel(int M, const unsigned long long *__restric
     }
 }
 
-typedef CUresult (*LmEncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                               const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                               CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-static LmEncodeFn lm_encode_fn() {
-    static LmEncodeFn fn = nullptr;
-    if (!fn) {
-        void *ptr = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<LmEncodeFn>(ptr);
-    }
-    return fn;
-}
-// [rows][H] bf16 row-major, box = 64 columns x box_rows rows, 128-byte swizzle
-static bool lm_map(CUtensorMap *map, const void *base, int rows, int H, int box_rows) {
-    LmEncodeFn fn = lm_encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)H, (cuuint64_t)rows};
-    const cuuint64_t str[1] = {(cuuint64_t)H * 2};
-    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-    const cuuint32_t ones[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, str, box, ones,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace mtv
 
 extern "C" int lm_head_argmax(const mtv_tree_t *tree, int B, int H, int V, const mtv_bf16 *x, const mtv_bf16 *W,
@@ -314,7 +288,7 @@ extern "C" int lm_head_argmax(const mtv_tree_t *tree, int B, int H, int V, const
     const int rounds = (min_pairs + ctas - 1) / ctas;
     p.n_pairs = ctas * rounds;
     p.R = ((V + 2 * p.n_pairs - 1) / (2 * p.n_pairs) + 7) / 8 * 8;
-    if (!lm_map(&w_map, W, V, H, p.R) || !lm_map(&x_map, x, M, H, N)) return MTV_ERR_CUDA;
+    if (!tma_map_2d_bf16(&w_map, W, V, H, p.R) || !tma_map_2d_bf16(&x_map, x, M, H, N)) return MTV_ERR_CUDA;
     const dim3 grid(passes, ctas);
     if (N == 64) lm_head_argmax_kernel<64><<<grid, LM_THREADS, smem, st>>>(w_map, x_map, p);
     else lm_head_argmax_kernel<128><<<grid, LM_THREADS, smem, st>>>(w_map, x_map, p);
