@@ -55,9 +55,9 @@ struct HeadsWs {
 HeadsWs heads_ws_layout(const mtv_tree *t, int B, int H, int V);
 bool heads_tc_eligible(int B, int H);
 size_t heads_tc_xsplit_bytes(int K, int H);
-int launch_heads_vocab_tc(const mtv_tree *t, int B, int H, int V, const __nv_bfloat16 *W2, const int32_t *root_tok,
-                          int32_t *cand, float *cand_logit, int32_t *tree_tok, const HeadsWs &L, char *ws,
-                          cudaStream_t st);
+int launch_heads_tc(const mtv_tree *t, int B, int H, int V, const __nv_bfloat16 *hidden, const __nv_bfloat16 *W1,
+                    const __nv_bfloat16 *b1, const __nv_bfloat16 *W2, const int32_t *root_tok, int32_t *cand,
+                    float *cand_logit, int32_t *tree_tok, const HeadsWs &L, char *ws, cudaStream_t st);
 
 struct AttnWs {
     size_t o_off, ml_off, total;

@@ -448,11 +448,8 @@ static int launch_heads(const mtv_tree *t, int B, int H, int V, const __nv_bfloa
     const int btiles = (B + NB - 1) / NB;
     const size_t sm1 = (size_t)NB * H * sizeof(float);
     const VocabSmem S = vocab_smem_plan(NB, H, L.ctas_per_head);
-    if (sm1 > VT_SMEM_MAX) return MTV_ERR_UNSUPPORTED_SHAPE;
-    if (!L.use_tc) {
-        if (S.total == 0) return MTV_ERR_UNSUPPORTED_SHAPE;
-        if (NB > 1 && S.rows_per_stage < (NB >= 4 ? 4 : 2)) return MTV_ERR_UNSUPPORTED_SHAPE;   // rows too long for a block of rows per stage
-    }
+    if (sm1 > VT_SMEM_MAX || S.total == 0) return MTV_ERR_UNSUPPORTED_SHAPE;
+    if (NB > 1 && S.rows_per_stage < (NB >= 4 ? 4 : 2)) return MTV_ERR_UNSUPPORTED_SHAPE;   // rows too long for a block of rows per stage
     static bool attr_done = false;
     if (!attr_done) {
         MTV_CUDA_CHECK(cudaFuncSetAttribute(heads_resblock_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, VT_SMEM_MAX));
@@ -468,7 +465,6 @@ static int launch_heads(const mtv_tree *t, int B, int H, int V, const __nv_bfloa
         heads_resblock_kernel<NB><<<dim3(g1, btiles), HEADS_THREADS, sm1, st>>>(B, H, t->K, hidden, W1, b1, hprime,
                                                                                counters, L.n_counters);
     }
-    if (L.use_tc) return launch_heads_vocab_tc(t, B, H, V, W2, root_tok, cand, cand_logit, tree_tok, L, ws, st);
     VocabParams p;
     p.B = B; p.H = H; p.V = V; p.K = t->K; p.T = t->T; p.C = t->C;
     p.W2 = W2; p.hprime = hprime;
@@ -510,7 +506,8 @@ extern "C" int medusa_heads_topk(const mtv_tree_t *tree, int B, int H, int V,
     auto *bb = reinterpret_cast<const __nv_bfloat16 *>(b1);
     auto *w2 = reinterpret_cast<const __nv_bfloat16 *>(W2);
     int rc;
-    if (B == 1) rc = launch_heads<1>(tree, B, H, V, h, w1, bb, w2, root_tok, cand, cand_logit, tree_tok, L, (char *)ws, st);
+    if (L.use_tc) rc = launch_heads_tc(tree, B, H, V, h, w1, bb, w2, root_tok, cand, cand_logit, tree_tok, L, (char *)ws, st);
+    else if (B == 1) rc = launch_heads<1>(tree, B, H, V, h, w1, bb, w2, root_tok, cand, cand_logit, tree_tok, L, (char *)ws, st);
     else if (B == 2) rc = launch_heads<2>(tree, B, H, V, h, w1, bb, w2, root_tok, cand, cand_logit, tree_tok, L, (char *)ws, st);
     else if (B <= 4) rc = launch_heads<4>(tree, B, H, V, h, w1, bb, w2, root_tok, cand, cand_logit, tree_tok, L, (char *)ws, st);
     else rc = launch_heads<8>(tree, B, H, V, h, w1, bb, w2, root_tok, cand, cand_logit, tree_tok, L, (char *)ws, st);

@@ -52,21 +52,185 @@ __device__ __forceinline__ void ht_tma_2d(uint32_t dst, const void *map, uint32_
                  ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
 
-// xsplit[k][part][b][o], part = 0 (hi), 1 (mid), 2 (lo): h' = hi + mid + lo up to 2^-25; rows b >= B are zero.
-__global__ void heads_split_kernel(int K, int B, int H, const float *__restrict__ hprime, __nv_bfloat16 *__restrict__ xsplit) {
-    const size_t n = (size_t)K * HT_NB * H;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        const int o = (int)(i % H), b = (int)((i / H) % HT_NB), k = (int)(i / ((size_t)H * HT_NB));
-        float x = b < B ? hprime[((size_t)k * B + b) * H + o] : 0.f;
-        const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-        x -= __bfloat162float(hi);                         // exact
-        const __nv_bfloat16 mid = __float2bfloat16_rn(x);
-        x -= __bfloat162float(mid);                        // exact
-        const __nv_bfloat16 lo = __float2bfloat16_rn(x);
-        __nv_bfloat16 *dst = xsplit + ((size_t)k * HT_N + b) * H + o;
-        dst[0] = hi;
-        dst[(size_t)HT_NB * H] = mid;
-        dst[(size_t)2 * HT_NB * H] = lo;
+// ---------------------------------------------------------------------------
+// Residual block for several batch rows:  h'[k][b][o] = h[b][o] + SiLU(W1[k][o][:] . h[b][:] + b1[k][o]).
+// The same pipeline with the K H rows of W1 as the MMA's M side (tiles of 128 rows, persistent CTAs) and the
+// bf16 hidden states of up to 16 batch rows as its N side (exact: they are bf16 to begin with).  The epilogue
+// (thread = output row) adds the four accumulators, the bias and the residual in fp32 and writes h' as the
+// three bf16 terms the vocabulary projection multiplies: xsplit[k][part][b][o], part = 0 (hi), 1 (mid),
+// 2 (lo), h' = hi + mid + lo up to 2^-25.  Batch rows b >= B hold finite values nobody reads.
+constexpr int RT_STAGES = 8;
+constexpr uint32_t RT_X_BYTES = HT_NB * 128;
+constexpr uint32_t RT_STAGE_BYTES = HT_W_BYTES + RT_X_BYTES;   // 18 KB
+constexpr uint32_t RT_SMEM_BYTES = 1024 + RT_STAGES * RT_STAGE_BYTES;
+constexpr uint32_t RT_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(HT_NB >> 3) << 17) | ((128u >> 4) << 24);
+static_assert(RT_STAGE_BYTES % 1024 == 0, "stages must keep the 1024-byte alignment of the swizzled tiles");
+
+struct ResblockTcParams {
+    int B, H, K;
+    const __nv_bfloat16 *hidden, *b1;
+    __nv_bfloat16 *xsplit;
+    int32_t *counters;
+    int n_counters;
+    int32_t *dev_error;
+};
+
+// w_map: [K H][H] rows of W1, box 64 x 128; h_map: [B][H] hidden states, box 64 x 16 (rows >= B read as zero).
+__global__ void __launch_bounds__(HT_THREADS, 1)
+heads_resblock_tc_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap h_map,
+                         const ResblockTcParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag_s;
+    __shared__ int issued_s;
+    __shared__ __align__(8) unsigned long long bar_mem[2 * RT_STAGES + 5];
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const uint32_t raw = ptx::smem_u32(smem_raw);
+    const uint32_t ring = raw + ((1024u - (raw & 1023u)) & 1023u);
+    const uint32_t bars = ptx::smem_u32(bar_mem);
+    auto full = [&](int s) { return bars + (uint32_t)s * 8u; };
+    auto empty = [&](int s) { return bars + (uint32_t)(RT_STAGES + s) * 8u; };
+    auto acc_full = [&](int u) { return bars + (uint32_t)(2 * RT_STAGES + u) * 8u; };
+    auto acc_empty = [&](int u) { return bars + (uint32_t)(2 * RT_STAGES + 2 + u) * 8u; };
+    const uint32_t drain_bar = bars + (uint32_t)(2 * RT_STAGES + 4) * 8u;
+    volatile int *abort_flag = &abort_flag_s;
+    constexpr uint32_t TMEM_COLS = 2 * HT_NACC * HT_NB;   // 128
+
+    // tickets of the vocabulary kernel (the next launch on the stream) start at zero
+    if (blockIdx.x == 0)
+        for (int i = threadIdx.x; i < p.n_counters; i += HT_THREADS) p.counters[i] = 0;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < RT_STAGES; ++s) { ptx::mbar_init(full(s), 1); ptx::mbar_init(empty(s), 1); }
+        for (int u = 0; u < 2; ++u) { ptx::mbar_init(acc_full(u), 1); ptx::mbar_init(acc_empty(u), 128); }
+        ptx::mbar_init(drain_bar, 1);
+        ptx::fence_mbar_init();
+        abort_flag_s = 0;
+        issued_s = 0;
+        ptx::prefetch_tensormap(&w_map);
+        ptx::prefetch_tensormap(&h_map);
+    }
+    if (warp == 4) {
+        ptx::tmem_alloc(ptx::smem_u32(&tmem_slot), TMEM_COLS);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+
+    const int rows = p.K * p.H;
+    const int n_tiles_all = (rows + 127) / 128;
+    const int my_tiles = (int)blockIdx.x < n_tiles_all ? (n_tiles_all - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+    const int n_kc = p.H / 64;
+
+    if (warp == 5) {
+        // ---------------------------------------------------------------- TMA producer
+        int it = 0;
+        for (int q = 0; q < my_tiles && !*abort_flag; ++q) {
+            const int row0 = ((int)blockIdx.x + q * (int)gridDim.x) * 128;
+            for (int kc = 0; kc < n_kc; ++kc, ++it) {
+                const int s = it % RT_STAGES, use = it / RT_STAGES;
+                if (use > 0 && !ptx::mbar_wait(empty(s), (use - 1) & 1)) { *abort_flag = 1; break; }
+                if (lane == 0) {
+                    const uint32_t base = ring + s * RT_STAGE_BYTES;
+                    ptx::mbar_arrive_expect_tx(full(s), RT_STAGE_BYTES);
+                    ht_tma_2d(base, &w_map, full(s), kc * 64, row0);
+                    ht_tma_2d(base + HT_W_BYTES, &h_map, full(s), kc * 64, 0);
+                }
+                __syncwarp();
+            }
+        }
+        if (lane == 0) issued_s = it;
+    } else if (warp == 4) {
+        // ---------------------------------------------------------------- MMA issuer
+        int it = 0;
+        bool ok = true;
+        for (int q = 0; ok && q < my_tiles && !*abort_flag; ++q) {
+            const int u = q & 1;
+            if (q >= 2) ok = ptx::mbar_wait(acc_empty(u), ((q >> 1) - 1) & 1);
+            if (!ok) break;
+            ptx::tc_fence_after();
+            for (int kc = 0; kc < n_kc; ++kc, ++it) {
+                const int s = it % RT_STAGES;
+                ok = ptx::mbar_wait(full(s), (it / RT_STAGES) & 1);
+                if (!ok) break;
+                ptx::tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t base = ring + s * RT_STAGE_BYTES;
+                    const uint32_t d = tmem + (u * HT_NACC + kc % HT_NACC) * HT_NB;
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        ptx::mma_ss(d, ht_desc(base + kk * 32), ht_desc(base + HT_W_BYTES + kk * 32), RT_IDESC,
+                                    kc >= HT_NACC || kk > 0);
+                    ptx::tc_commit(empty(s));
+                    if (kc == n_kc - 1) ptx::tc_commit(acc_full(u));
+                }
+                __syncwarp();
+            }
+        }
+        if (!ok) *abort_flag = 1;
+    } else {
+        // ---------------------------------------------------------------- epilogue: thread = output row
+        const int n_acc = min(HT_NACC, n_kc);
+        bool ok = true;
+        for (int q = 0; q < my_tiles; ++q) {
+            const int u = q & 1;
+            if (*abort_flag) ok = false;
+            if (ok) ok = ptx::mbar_wait(acc_full(u), (q >> 1) & 1);
+            __syncwarp();
+            ptx::tc_fence_after();
+            float y[HT_NB];
+#pragma unroll
+            for (int b = 0; b < HT_NB; ++b) y[b] = 0.f;
+            for (int a = 0; a < n_acc; ++a) {
+                uint32_t acc[16];
+                ptx::tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (u * HT_NACC + a) * HT_NB, acc);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int b = 0; b < HT_NB; ++b) y[b] += __uint_as_float(acc[b]);
+            }
+            ptx::tc_fence_before();
+            ptx::mbar_arrive(acc_empty(u));
+            const int r = ((int)blockIdx.x + q * (int)gridDim.x) * 128 + warp * 32 + lane;
+            if (ok && r < rows) {
+                const int k = r / p.H, o = r % p.H;
+                const float bias = p.b1 ? __bfloat162float(p.b1[(size_t)k * p.H + o]) : 0.f;
+#pragma unroll
+                for (int b = 0; b < HT_NB; ++b) {
+                    const float yy = y[b] + bias;
+                    const float h = b < p.B ? __bfloat162float(p.hidden[(size_t)b * p.H + o]) : 0.f;
+                    float x = h + yy / (1.f + expf(-yy));
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+                    x -= __bfloat162float(hi);                         // exact
+                    const __nv_bfloat16 mid = __float2bfloat16_rn(x);
+                    x -= __bfloat162float(mid);                        // exact
+                    __nv_bfloat16 *dst = p.xsplit + ((size_t)k * HT_N + b) * p.H + o;
+                    dst[0] = hi;
+                    dst[(size_t)HT_NB * p.H] = mid;
+                    dst[(size_t)2 * HT_NB * p.H] = __float2bfloat16_rn(x);
+                }
+            }
+        }
+        if (!ok) *abort_flag = 1;
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 4) {
+        if (*abort_flag) {
+            if (lane == 0) ptx::tc_commit(drain_bar);
+            __syncwarp();
+            ptx::mbar_wait(drain_bar, 0);
+        }
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem, TMEM_COLS);
+    }
+    if (*abort_flag) {
+        if (threadIdx.x == 0) atomicExch(p.dev_error, MTV_ERR_TIMEOUT);
+        if (warp == 5 && lane == 0)
+            for (int s = 0; s < RT_STAGES; ++s) {
+                const int uses = (issued_s - s + RT_STAGES - 1) / RT_STAGES;
+                if (issued_s > s) ptx::mbar_wait(full(s), (uses - 1) & 1);
+            }
     }
 }
 
@@ -256,23 +420,34 @@ bool heads_tc_eligible(int B, int H) { return B >= 2 && B <= HT_NB && H >= 64 &&
 
 size_t heads_tc_xsplit_bytes(int K, int H) { return (size_t)K * HT_N * H * sizeof(__nv_bfloat16); }
 
-// hprime -> split activations -> projection, top-k, merges, tree expansion.  The residual block has run.
-int launch_heads_vocab_tc(const mtv_tree *t, int B, int H, int V, const __nv_bfloat16 *W2, const int32_t *root_tok,
-                          int32_t *cand, float *cand_logit, int32_t *tree_tok, const HeadsWs &L, char *ws,
-                          cudaStream_t st) {
+// Residual block, then projection, top-k, merges and tree expansion: the whole medusa_heads_topk for 2..16 rows.
+int launch_heads_tc(const mtv_tree *t, int B, int H, int V, const __nv_bfloat16 *hidden, const __nv_bfloat16 *W1,
+                    const __nv_bfloat16 *b1, const __nv_bfloat16 *W2, const int32_t *root_tok, int32_t *cand,
+                    float *cand_logit, int32_t *tree_tok, const HeadsWs &L, char *ws, cudaStream_t st) {
     static bool attr_done = false;
     if (!attr_done) {
         MTV_CUDA_CHECK(cudaFuncSetAttribute(heads_vocab_topk_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, HT_SMEM_BYTES));
+        MTV_CUDA_CHECK(cudaFuncSetAttribute(heads_resblock_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, RT_SMEM_BYTES));
         attr_done = true;
     }
-    const float *hprime = reinterpret_cast<const float *>(ws + L.hprime_off);
     __nv_bfloat16 *xsplit = reinterpret_cast<__nv_bfloat16 *>(ws + L.xsplit_off);
-    CUtensorMap w_map, x_map;
-    if (!tma_map_2d_bf16(&w_map, W2, t->K * V, H, 128) || !tma_map_2d_bf16(&x_map, xsplit, t->K * HT_N, H, HT_N))
+    CUtensorMap w1_map, h_map, w2_map, x_map;
+    if (!tma_map_2d_bf16(&w1_map, W1, t->K * H, H, 128) || !tma_map_2d_bf16(&h_map, hidden, B, H, HT_NB) ||
+        !tma_map_2d_bf16(&w2_map, W2, t->K * V, H, 128) || !tma_map_2d_bf16(&x_map, xsplit, t->K * HT_N, H, HT_N))
         return MTV_ERR_CUDA;
+    {
+        ResblockTcParams r;
+        r.B = B; r.H = H; r.K = t->K; r.hidden = hidden; r.b1 = b1; r.xsplit = xsplit;
+        r.counters = reinterpret_cast<int32_t *>(ws + L.counters_off); r.n_counters = L.n_counters;
+        r.dev_error = t->d_error;
+        int ctas = (t->K * H + 127) / 128;
+        if (ctas > sm_count()) ctas = sm_count();
+        TapScope tap(MTV_KERNEL_HEADS_RESBLOCK, st);
+        heads_resblock_tc_kernel<<<ctas, HT_THREADS, RT_SMEM_BYTES, st>>>(w1_map, h_map, r);
+    }
     VocabParams p;
     p.B = B; p.H = H; p.V = V; p.K = t->K; p.T = t->T; p.C = t->C;
-    p.W2 = W2; p.hprime = hprime;
+    p.W2 = W2; p.hprime = nullptr;
     p.kd_arr = t->d_kd; p.off_arr = t->d_cand_offset; p.tree_indices = t->d_tree_indices; p.root_tok = root_tok;
     p.part_val = reinterpret_cast<float *>(ws + L.part_val_off);
     p.part_idx = reinterpret_cast<int32_t *>(ws + L.part_idx_off);
@@ -282,9 +457,7 @@ int launch_heads_vocab_tc(const mtv_tree *t, int B, int H, int V, const __nv_bfl
     p.rows_per_stage = 0; p.n_stages = 0; p.n_it = 0;
     p.stage_bytes = 0; p.xs_off = 0; p.lists_off = 0; p.zbuf_off = 0; p.bars_off = 0;
     TapScope tap(MTV_KERNEL_HEADS_VOCAB_TOPK, st);
-    const size_t n = (size_t)t->K * HT_NB * H;
-    heads_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(t->K, B, H, hprime, xsplit);
-    heads_vocab_topk_tc_kernel<<<dim3(L.ctas_per_head, t->K), HT_THREADS, HT_SMEM_BYTES, st>>>(w_map, x_map, p);
+    heads_vocab_topk_tc_kernel<<<dim3(L.ctas_per_head, t->K), HT_THREADS, HT_SMEM_BYTES, st>>>(w2_map, x_map, p);
     return MTV_OK;
 }
 
