@@ -111,6 +111,15 @@ def test_attention_ragged_batch_many_splits_and_strided_cache():
     _attention_case(tb, tree, 3, 8, 2, 128, [1500, 40, 777], seed=9, Lcap=1600, pad=24)
 
 
+def test_attention_large_ragged_batch():
+    """More query blocks than half the SMs: one CTA per block and no key splits, sequences from empty to full."""
+    tb, tree = make_tree("rank_prior", 4, (), 64)
+    g = torch.Generator().manual_seed(77)
+    lens = torch.randint(0, 1100, (40,), generator=g).tolist()
+    lens[3], lens[17] = 0, 1099
+    _attention_case(tb, tree, 40, 8, 2, 128, lens, seed=12, Lcap=1100 + tree.T)
+
+
 @pytest.mark.parametrize("D", [64, 128])
 def test_attention_capacity_is_reported_not_faulted(D):
     tb, tree = make_tree("cartesian", 2, (2, 2))
