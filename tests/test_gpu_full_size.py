@@ -46,7 +46,7 @@ def test_attention_full_size_sampled_rows(name, n_rows):
     assert out.float().abs().max().item() <= vmax * 1.01 and bool(torch.isfinite(out.float()).all())
 
 
-@pytest.mark.parametrize("name,rows", [("long", None), ("batched", [0, 9, 15])])
+@pytest.mark.parametrize("name,rows", [("long", None), ("batched", [0, 9, 15]), ("stress", [2])])
 def test_heads_full_size(name, rows):
     w = synth.WORKLOADS[name]
     tb, tree = workload_tree(w)
@@ -126,7 +126,7 @@ def test_attention_is_bitwise_repeatable(name, reps):
 def test_heads_are_bitwise_repeatable():
     w = synth.WORKLOADS["long"]
     tb, tree = workload_tree(w)
-    hidden, W1, b1, W2, root = synth.head_inputs(4, w.H, 32768, w.K, 99, device=DEV)    # the 4-row (blocked) path
+    hidden, W1, b1, W2, root = synth.head_inputs(4, w.H, 32768, w.K, 99, device=DEV)    # four rows: the tensor-core path
     ws = workspace(tree, 4, w.H, 32768, 0, 0, 0, 0)
     ref_c = torch.zeros(4, tree.C, dtype=torch.int32, device=DEV)
     ref_l = torch.zeros(4, tree.C - 1, device=DEV)
