@@ -228,7 +228,6 @@ __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
             while (ld_acquire(p.arrive + grp) < nsplit)
                 if (clock64() - t0 > ptx::WAIT_CYCLE_LIMIT) { atomicExch(p.dev_error, MTV_ERR_TIMEOUT); break; }
             TRACE(53);   // everybody arrived
-            ptx::fence_proxy_async_all();
         }
         cta_sync();
         // ---- fetch rows [row_begin, row_begin + n_my) of every split: one bulk copy per split, one lane each
