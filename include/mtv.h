@@ -11,7 +11,11 @@
  *                          tokens through retrieve_indices
  *   kv_compact_accepted    the same Gather applied to the accepted nodes' K/V rows,
  *                          in place, all layers; advances seq_lens
- * with the tree's static tensors built once by tree_build_static.
+ * with the tree's static tensors built once by tree_build_static.  Beside the step proper:
+ *   tree_kv_append_rope    K/V rows of the tree nodes into the cache, rotary embedding at
+ *                          position seq_len + depth
+ *   lm_head_argmax         the base model's LM head with the per-node argmax fused in, and
+ *   tree_accept_keys       the acceptance that reads its result instead of stored logits
  *
  * Conventions
  *   - Every function returns an int: MTV_OK (0) or a negative MTV_ERR_* code.
@@ -27,7 +31,8 @@
  *     the caller's device `status[B]` (0 = ok, MTV_ERR_* otherwise); the outputs of
  *     that sequence are left untouched.  status may be NULL.
  *   - Supported shapes: D in {64, 128}; 1 <= T <= 128; 1 <= K <= 8; per-depth
- *     top-k <= 16; Hq a multiple of Hkv with Hq/Hkv <= 8; H a multiple of 8.
+ *     top-k <= 16; Hq a multiple of Hkv with Hq/Hkv <= 8; H a multiple of 8; at most
+ *     16 batch rows in medusa_heads_topk.
  *     Anything else returns MTV_ERR_UNSUPPORTED_SHAPE.
  */
 #ifndef MTV_H_
