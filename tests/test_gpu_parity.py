@@ -26,6 +26,10 @@ HEAD_CASES = [
     (5, 1024, 5000, 4, ("rank_prior", (), 64)),
     (16, 512, 2048, 2, ("cartesian", (16, 3), 0)),
     (1, 8, 20, 1, ("cartesian", (16,), 0)),               # V barely above top-k
+    (2, 512, 2048, 3, ("cartesian", (4, 2, 2), 0)),       # two rows, H a multiple of 64: the tensor-core kernels
+    (9, 256, 3001, 4, ("rank_prior", (), 64)),            # an odd number of rows above 8
+    (4, 64, 50, 1, ("cartesian", (16,), 0)),              # one K chunk, slabs far shorter than a 128-row tile
+    (16, 192, 777, 5, ("rank_prior", (), 128)),           # three K chunks (fewer than the four accumulators)
 ]
 
 
