@@ -336,6 +336,13 @@ int mtv_kernel_taps_used(int kernel_id);
  * synchronises with the device: use it between steps, not inside one. */
 int mtv_device_error(const mtv_tree_t *tree, int clear, int32_t *code);
 
+/* Self-test of that mechanism (the paper has no counterpart): one warp waits, with the same
+ * bounded wait the hot kernels use, on a shared-memory barrier that nothing ever arrives on.
+ * After about a second of SM cycles the wait gives up, the kernel stores MTV_ERR_TIMEOUT in the
+ * tree's device error word and returns normally: nothing faults, the context stays usable.
+ * Only enqueues the kernel; read the word with mtv_device_error afterwards. */
+int mtv_selftest_wait_timeout(const mtv_tree_t *tree, void *stream);
+
 /* Human-readable text for the most recent MTV_ERR_CUDA (or refused size) on this thread (never NULL). */
 const char *mtv_last_error(void);
 

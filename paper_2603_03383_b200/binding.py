@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libmtv.so")
 MTV_OK = 0
 ERR = {-1: "MTV_ERR_INVALID_ARG", -2: "MTV_ERR_UNSUPPORTED_SHAPE", -3: "MTV_ERR_WORKSPACE",
        -4: "MTV_ERR_CUDA", -5: "MTV_ERR_TIMEOUT", -6: "MTV_ERR_CAPACITY"}
+MTV_ERR_TIMEOUT = -5
 MTV_ERR_CAPACITY = -6
 MAX_K = 8
 
@@ -27,7 +28,7 @@ EXPORTS = ["tree_build_static", "tree_gen_cartesian", "tree_gen_rank_prior", "tr
            "kv_compact_accepted", "mtv_verify_step", "mtv_verify_step_host", "mtv_last_error",
            "mtv_set_kernel_taps", "mtv_kernel_taps_used", "mtv_device_error",
            "tree_accept_static_scratch", "tree_accept_static_scratch_capacity", "tree_kv_append_rope",
-           "lm_head_argmax", "tree_accept_keys"]
+           "lm_head_argmax", "tree_accept_keys", "mtv_selftest_wait_timeout"]
 
 
 class MtvError(RuntimeError):
@@ -104,6 +105,7 @@ def lib():
                                           vp, vp]
         L.lm_head_argmax.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         L.tree_accept_keys.argtypes = [vp, i32] + [vp] * 7 + [vp]
+        L.mtv_selftest_wait_timeout.argtypes = [vp, vp]
         _lib = L
     return _lib
 
@@ -183,6 +185,11 @@ def mtv_device_error(tree: Tree, clear: bool = True) -> int:
     code = C.c_int32(0)
     _check(lib().mtv_device_error(tree.handle, 1 if clear else 0, C.byref(code)), "mtv_device_error")
     return code.value
+
+
+def mtv_selftest_wait_timeout(tree: Tree, stream=None):
+    """Enqueue a kernel whose bounded wait must run out (about a second); see include/mtv.h."""
+    _check(lib().mtv_selftest_wait_timeout(tree.handle, _stream(stream)), "mtv_selftest_wait_timeout")
 
 
 def mtv_workspace_bytes(tree: Tree, B, H, V, Hq, Hkv, D, Lcap) -> int:

@@ -1,5 +1,6 @@
 // Whole verification step on one stream, and its host-buffer variant.
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 extern "C" size_t mtv_workspace_bytes(const mtv_tree_t *tree, int B, int H, int V, int Hq, int Hkv, int D, int Lcap) {
     using namespace mtv;
@@ -133,5 +134,28 @@ extern "C" int mtv_verify_step_host(const mtv_tree_t *tree, const mtv_step_args 
     MTV_CUDA_CHECK(cudaEventRecord(g_aux.down_done, down));
     MTV_CUDA_CHECK(cudaStreamWaitEvent(st, g_aux.down_done, 0));
     MTV_CUDA_CHECK(cudaStreamSynchronize(st));
+    return MTV_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Self-test of the bounded waits: a barrier nobody arrives on.
+namespace {
+__global__ void selftest_wait_timeout_kernel(int32_t *dev_error) {
+    __shared__ __align__(8) unsigned long long bar_mem;
+    const uint32_t bar = mtv::ptx::smem_u32(&bar_mem);
+    if (threadIdx.x == 0) {
+        mtv::ptx::mbar_init(bar, 1);
+        mtv::ptx::fence_mbar_init();
+    }
+    __syncwarp();
+    const bool ok = mtv::ptx::mbar_wait(bar, 0);      // gives up after WAIT_CYCLE_LIMIT cycles
+    if (!ok && threadIdx.x == 0) atomicExch(dev_error, MTV_ERR_TIMEOUT);
+}
+}  // namespace
+
+extern "C" int mtv_selftest_wait_timeout(const mtv_tree_t *tree, void *stream) {
+    if (!tree || !tree->on_device) return MTV_ERR_INVALID_ARG;
+    selftest_wait_timeout_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(tree->d_error);
+    MTV_CUDA_CHECK(cudaGetLastError());
     return MTV_OK;
 }

@@ -466,3 +466,18 @@ def test_tree_kv_append_rope_capacity():
     torch.cuda.synchronize()
     assert status.tolist() == [binding.MTV_ERR_CAPACITY, 0]
     assert torch.equal(q[0], q0[0]) and not torch.equal(q[1], q0[1]) and bool((kc[0] == 0).all())
+
+
+# ------------------------------------------------------- failure detection
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    """No fault is provoked: a barrier nobody arrives on makes the kernels' bounded wait give up after about a
+    second; the error word says so, clearing it works, and the next hot call runs and matches the oracle."""
+    tb, tree = make_tree("cartesian", 2, (2, 2))
+    assert binding.mtv_device_error(tree) == 0
+    binding.mtv_selftest_wait_timeout(tree)
+    torch.cuda.synchronize()
+    assert binding.mtv_device_error(tree, clear=False) == binding.MTV_ERR_TIMEOUT     # sticky until cleared
+    assert binding.mtv_device_error(tree) == binding.MTV_ERR_TIMEOUT
+    assert binding.mtv_device_error(tree) == 0
+    _attention_case(tb, tree, 1, 8, 2, 128, [300], seed=3)
+    assert binding.mtv_device_error(tree) == 0
