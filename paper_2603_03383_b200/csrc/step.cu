@@ -55,7 +55,7 @@ namespace {
 struct HostStepAux {
     cudaStream_t up = nullptr, down = nullptr;
     cudaEvent_t start = nullptr, q_up = nullptr, logits_up = nullptr, down_done = nullptr;
-    cudaEvent_t chunk[4] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t chunk[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     bool ready = false;
 };
 HostStepAux g_aux;
@@ -64,7 +64,7 @@ int host_step_aux() {
     MTV_CUDA_CHECK(cudaStreamCreateWithFlags(&g_aux.up, cudaStreamNonBlocking));
     MTV_CUDA_CHECK(cudaStreamCreateWithFlags(&g_aux.down, cudaStreamNonBlocking));
     cudaEvent_t *ev[] = {&g_aux.start, &g_aux.q_up, &g_aux.logits_up, &g_aux.down_done, &g_aux.chunk[0], &g_aux.chunk[1],
-                         &g_aux.chunk[2], &g_aux.chunk[3]};
+                         &g_aux.chunk[2], &g_aux.chunk[3], &g_aux.chunk[4], &g_aux.chunk[5], &g_aux.chunk[6], &g_aux.chunk[7]};
     for (cudaEvent_t *e : ev) MTV_CUDA_CHECK(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
     g_aux.ready = true;
     return MTV_OK;
@@ -73,7 +73,7 @@ int host_step_aux() {
 
 // The transfers overlap the compute: the queries and the base-model logits go up on a copy stream while the
 // heads run (attention waits for the queries, acceptance for the logits), and the attention outputs come
-// down on a second copy stream in up to four groups of layers while later layers are still running.
+// down on a second copy stream in up to sixteen groups of layers while later layers are still running.
 extern "C" int mtv_verify_step_host(const mtv_tree_t *tree, const mtv_step_args *d, const mtv_step_args *h,
                                     void *stream) {
     if (!tree || !d || !h || !d->k_caches_host || !d->v_caches_host) return MTV_ERR_INVALID_ARG;
@@ -102,7 +102,7 @@ extern "C" int mtv_verify_step_host(const mtv_tree_t *tree, const mtv_step_args 
     MTV_CUDA_CHECK(cudaMemcpyAsync(h->tree_tok, d->tree_tok, B * T * 4, cudaMemcpyDeviceToHost, st));
     // attention, its outputs leaving in groups of layers
     MTV_CUDA_CHECK(cudaStreamWaitEvent(st, g_aux.q_up, 0));
-    const int per_group = (d->n_layers + 3) / 4;
+    const int per_group = (d->n_layers + 15) / 16;
     int sent = 0, n_sent = 0;
     for (int l = 0; l < d->n_layers; ++l) {
         rc = tree_verify_attention(tree, d->B, d->Hq, d->Hkv, d->D, d->q_layers + l * per_layer, d->k_caches_host[l],
@@ -110,7 +110,7 @@ extern "C" int mtv_verify_step_host(const mtv_tree_t *tree, const mtv_step_args 
                                    d->scale, d->out_layers + l * per_layer, d->status, d->ws, d->ws_bytes, stream);
         if (rc != MTV_OK) return rc;
         if ((l + 1) % per_group == 0 || l + 1 == d->n_layers) {
-            cudaEvent_t ev = g_aux.chunk[n_sent++ % 4];
+            cudaEvent_t ev = g_aux.chunk[n_sent++ % 8];
             MTV_CUDA_CHECK(cudaEventRecord(ev, st));
             MTV_CUDA_CHECK(cudaStreamWaitEvent(down, ev, 0));
             MTV_CUDA_CHECK(cudaMemcpyAsync(h->out_layers + sent * per_layer, d->out_layers + sent * per_layer,
