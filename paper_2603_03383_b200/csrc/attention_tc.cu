@@ -24,7 +24,7 @@
 // (plain loads would be throttled by the little L1 this kernel leaves), combines them in fp32 with
 // the weights exp2(m_s - m) l_s / sum and writes bf16 output rows.  The grid never exceeds one CTA per SM, so all CTAs are resident together and
 // the wait on the counter always ends; it is bounded all the same.  The counters live in the
-// tree object, start at zero and are put back to zero by the last CTA to leave.
+// tree object, start at zero and are put back to zero by the last CTA that has seen them full.
 //
 // The running max is only raised when the new row max exceeds it by more than 8 (in log2
 // units), so O in tensor memory is rescaled rarely; P stays below 2^8.
@@ -220,7 +220,7 @@ __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
             ptx::bulk_commit();
             ptx::bulk_wait_all();
             TRACE(51);   // partial left shared memory and is written
-            ptx::fence_proxy_async_all();
+            ptx::fence_proxy_async_global();
             // release-arrive without waiting for the counter's old value
             asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(p.arrive + grp) : "memory");
             TRACE(52);   // arrived
@@ -228,13 +228,20 @@ __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
             while (ld_acquire(p.arrive + grp) < nsplit)
                 if (clock64() - t0 > ptx::WAIT_CYCLE_LIMIT) { atomicExch(p.dev_error, MTV_ERR_TIMEOUT); break; }
             TRACE(53);   // everybody arrived
+            // Nobody polls the arrival counter once all have seen it full: the last one to get here puts both
+            // counters back to zero (the next call cannot start before this kernel has ended).
+            if (atomicAdd(p.depart + grp, 1) == nsplit - 1) {
+                p.arrive[grp] = 0;
+                p.depart[grp] = 0;
+                __threadfence();
+            }
         }
         cta_sync();
         // ---- fetch rows [row_begin, row_begin + n_my) of every split: one bulk copy per split, one lane each
         if (warp == 0 && n_my > 0) {
             if (lane == 0) ptx::mbar_arrive_expect_tx(bar(BAR_MERGE), (uint32_t)(nsplit * n_my) * TC_ROW_BYTES);
             __syncwarp();
-            ptx::fence_proxy_async_all();   // the other CTAs' partials, acquired above, before the async-proxy reads
+            ptx::fence_proxy_async_global();   // the other CTAs' partials, acquired above, before the async-proxy reads
             if (lane < nsplit)
                 ptx::bulk_g2s(ptx::smem_u32(c.tiles) + (uint32_t)(lane * n_my) * TC_ROW_BYTES,
                               p.ws_o + ((slab0 + lane) * 256 + row_begin) * 128, (uint32_t)n_my * TC_ROW_BYTES, bar(BAR_MERGE));
@@ -281,12 +288,6 @@ __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
                                         pack2_bf16(acc[4], acc[5]), pack2_bf16(acc[6], acc[7]));
         }
         if (warp == 0) TRACE(46);   // merge done
-        // the last CTA of the query block to get here puts the counters back to zero
-        if (threadIdx.x == 0 && atomicAdd(p.depart + grp, 1) == nsplit - 1) {
-            p.arrive[grp] = 0;
-            p.depart[grp] = 0;
-            __threadfence();
-        }
     }
     if (!SOFTMAX && warp == TC_MMA_WARP) {
         ptx::tc_fence_after();
