@@ -228,13 +228,6 @@ __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
             while (ld_acquire(p.arrive + grp) < nsplit)
                 if (clock64() - t0 > ptx::WAIT_CYCLE_LIMIT) { atomicExch(p.dev_error, MTV_ERR_TIMEOUT); break; }
             TRACE(53);   // everybody arrived
-            // Nobody polls the arrival counter once all have seen it full: the last one to get here puts both
-            // counters back to zero (the next call cannot start before this kernel has ended).
-            if (atomicAdd(p.depart + grp, 1) == nsplit - 1) {
-                p.arrive[grp] = 0;
-                p.depart[grp] = 0;
-                __threadfence();
-            }
         }
         cta_sync();
         // ---- fetch rows [row_begin, row_begin + n_my) of every split: one bulk copy per split, one lane each
@@ -247,6 +240,14 @@ __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
                               p.ws_o + ((slab0 + lane) * 256 + row_begin) * 128, (uint32_t)n_my * TC_ROW_BYTES, bar(BAR_MERGE));
         }
         if (warp == 0) TRACE(45);   // all splits arrived, rows on their way
+        // Nobody polls the arrival counter once all have seen it full: the last one to get here puts both counters
+        // back to zero (the next call cannot start before this kernel has ended).  Done here, behind the copies,
+        // so that the round trip of the atomic is not on the way of anything.
+        if (threadIdx.x == 0 && atomicAdd(p.depart + grp, 1) == nsplit - 1) {
+            p.arrive[grp] = 0;
+            p.depart[grp] = 0;
+            __threadfence();
+        }
         // ---- merge weights, one warp per row, lane s = split s: exp2(m_s - m) l_s / sum over the splits
         //      (split s contributes its own normalised result O_s / l_s)
         for (int rl = warp; rl < n_my; rl += TC_THREADS / 32) {
