@@ -230,14 +230,14 @@ __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
             TRACE(53);   // everybody arrived
         }
         cta_sync();
-        // ---- fetch rows [row_begin, row_begin + n_my) of every split: one bulk copy per split, one lane each
-        if (warp == 0 && n_my > 0) {
-            if (lane == 0) ptx::mbar_arrive_expect_tx(bar(BAR_MERGE), (uint32_t)(nsplit * n_my) * TC_ROW_BYTES);
-            __syncwarp();
+        // ---- fetch rows [row_begin, row_begin + n_my) of every split: one bulk copy per split, each issued by a
+        //      different warp (the copies of one warp's lanes are issued one after the other)
+        if (n_my > 0 && lane == 0) {
+            if (warp == 0) ptx::mbar_arrive_expect_tx(bar(BAR_MERGE), (uint32_t)(nsplit * n_my) * TC_ROW_BYTES);
             ptx::fence_proxy_async_global();   // the other CTAs' partials, acquired above, before the async-proxy reads
-            if (lane < nsplit)
-                ptx::bulk_g2s(ptx::smem_u32(c.tiles) + (uint32_t)(lane * n_my) * TC_ROW_BYTES,
-                              p.ws_o + ((slab0 + lane) * 256 + row_begin) * 128, (uint32_t)n_my * TC_ROW_BYTES, bar(BAR_MERGE));
+            for (int sp = warp; sp < nsplit; sp += TC_THREADS / 32)
+                ptx::bulk_g2s(ptx::smem_u32(c.tiles) + (uint32_t)(sp * n_my) * TC_ROW_BYTES,
+                              p.ws_o + ((slab0 + sp) * 256 + row_begin) * 128, (uint32_t)n_my * TC_ROW_BYTES, bar(BAR_MERGE));
         }
         if (warp == 0) TRACE(45);   // all splits arrived, rows on their way
         // Nobody polls the arrival counter once all have seen it full: the last one to get here puts both counters
