@@ -10,8 +10,11 @@
 // One persistent CTA per SM walks pairs of vocabulary tiles, so that a chunk of X fetched from L2
 // serves two weight tiles.  A tile holds R <= 128 rows, R chosen by the host so that every CTA gets
 // the same number of pairs (V = 32000 on 148 SMs: 112 rows); the MMA spans 128 rows all the same and
-// the rows past R, whatever the shared memory held, are left out of the maximum.  Warp roles: TMA producer (ring of stages, one stage = 64
-// columns of 256 weight rows and of the N node rows), MMA issuer (accumulators in tensor memory,
+// the rows past R, whatever the shared memory held, are left out of the maximum.  From 129 nodes up a
+// pass takes 256 nodes and one weight tile per stage: 128 x 256 x 16 is the MMA shape that runs at the
+// full tensor rate (128 x 128 x 16 reaches about 60 % of it), and the large batches are tensor-bound.
+// Warp roles: TMA producer (ring of stages, one stage = 64
+// columns of the weight tiles and of the N node rows), MMA issuer (accumulators in tensor memory,
 // double-buffered: the epilogue of one pair overlaps the MMAs of the next), four epilogue warps
 // (one thread per vocabulary row: order-preserving (value, ~index) keys, butterfly max over the
 // warp's 32 rows, shared-memory max across warps and pairs, one 64-bit atomic max per node at the end).
@@ -25,7 +28,7 @@ namespace mtv {
 
 constexpr int LM_THREADS = 192;            // warps 0-3 epilogue, warp 4 MMA issuer, warp 5 TMA producer
 constexpr int LM_KC = 64;                  // columns per stage: one 128-byte swizzle span
-constexpr uint32_t LM_W_BYTES = 256 * 128; // 256 weight rows x 64 columns
+constexpr uint32_t LM_TILE_BYTES = 128 * 128; // one weight tile of a stage: 128 rows x 64 columns
 constexpr uint32_t LM_SMEM_MAX = 220 * 1024;   // dynamic part; the static part (keys, barriers) is about 1.2 KB
 constexpr int LM_MAX_STAGES = 6;
 
@@ -34,10 +37,10 @@ constexpr uint32_t LM_IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >
 struct LmParams {
     unsigned long long *keys;   // [M] best (value, ~index) per node, zero before the launch
     int32_t *dev_error;
-    int M, H, V, N;             // N = nodes per pass (64 or 128)
+    int M, H, V, N;             // N = nodes per pass (64, 128 or 256)
     int R;                      // vocabulary rows per tile (<= 128, a multiple of 8), chosen so that the tiles
                                 // divide evenly among the CTAs; the MMA still spans 128 rows, the rest is ignored
-    int n_pairs;                // tile pairs over the vocabulary
+    int n_pairs;                // units (of two weight tiles, or of one when N = 256) over the vocabulary
     int n_stages;
     uint32_t stage_bytes;
 };
@@ -81,7 +84,9 @@ __device__ __forceinline__ unsigned long long warp_max_scatter32(unsigned long l
     return v[0];
 }
 
-template <int N>   // nodes per pass
+// N nodes per pass; TILES weight tiles per stage (2 for N <= 128, so that an X chunk serves two tiles; 1 for N = 256,
+// the MMA shape that runs at the full tensor rate, where two tiles' accumulators would not fit tensor memory twice)
+template <int N>
 __global__ void __launch_bounds__(LM_THREADS, 1)
 lm_head_argmax_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map,
                       const LmParams p) {
@@ -102,7 +107,9 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_co
     auto acc_empty = [&](int u) { return bars + (uint32_t)(2 * LM_MAX_STAGES + 2 + u) * 8u; };
     const uint32_t drain_bar = bars + (uint32_t)(2 * LM_MAX_STAGES + 4) * 8u;
     volatile int *abort_flag = &abort_flag_s;
-    constexpr uint32_t TMEM_COLS = 4 * N;   // 2 buffers x 2 tiles x N columns (256 or 512)
+    constexpr int TILES = N <= 128 ? 2 : 1;
+    constexpr uint32_t W_BYTES = TILES * LM_TILE_BYTES;
+    constexpr uint32_t TMEM_COLS = 2 * TILES * N;   // 2 buffers x TILES x N columns (256 or 512)
 
     for (int i = threadIdx.x; i < N; i += LM_THREADS) best[i] = 0ull;
     if (threadIdx.x == 0) {
@@ -131,21 +138,21 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_co
     const int n_pairs = p.n_pairs, R = p.R;
     const int my_pairs = cta < n_pairs ? (n_pairs - cta + n_cta - 1) / n_cta : 0;
     const int n_kc = p.H / LM_KC;
-    const uint32_t x_off = LM_W_BYTES;                   // X chunk sits after the weight chunk in a stage
+    const uint32_t x_off = W_BYTES;                      // X chunk sits after the weight chunk in a stage
 
     if (warp == 5) {
         // ---------------------------------------------------------------- TMA producer
         int it = 0;
         for (int q = 0; q < my_pairs && !*abort_flag; ++q) {
-            const int row0 = (cta + q * n_cta) * 2 * R;
+            const int row0 = (cta + q * n_cta) * TILES * R;
             for (int kc = 0; kc < n_kc; ++kc, ++it) {
                 const int s = it % NST, use = it / NST;
                 if (use > 0 && !ptx::mbar_wait(empty(s), (use - 1) & 1)) { *abort_flag = 1; break; }
                 if (lane == 0) {
                     const uint32_t base = ring + s * p.stage_bytes;
-                    ptx::mbar_arrive_expect_tx(full(s), (uint32_t)(2 * R + N) * 128u);
+                    ptx::mbar_arrive_expect_tx(full(s), (uint32_t)(TILES * R + N) * 128u);
                     tma_load_2d(base, &w_map, full(s), kc * LM_KC, row0);                 // rows past V arrive as zeros
-                    tma_load_2d(base + LM_W_BYTES / 2, &w_map, full(s), kc * LM_KC, row0 + R);
+                    if (TILES == 2) tma_load_2d(base + LM_TILE_BYTES, &w_map, full(s), kc * LM_KC, row0 + R);
                     tma_load_2d(base + x_off, &x_map, full(s), kc * LM_KC, pass * N);      // rows past M arrive as zeros
                 }
                 __syncwarp();
@@ -170,10 +177,10 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_co
                 if (lane == 0) {
                     const uint32_t base = ring + s * p.stage_bytes;
 #pragma unroll
-                    for (int t = 0; t < 2; ++t)
+                    for (int t = 0; t < TILES; ++t)
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk)
-                            ptx::mma_ss(tmem + (u * 2 + t) * N, lm_desc(base + t * (LM_W_BYTES / 2) + kk * 32),
+                            ptx::mma_ss(tmem + (u * TILES + t) * N, lm_desc(base + t * LM_TILE_BYTES + kk * 32),
                                         lm_desc(base + x_off + kk * 32), IDESC, kc > 0 || kk > 0);
                     ptx::tc_commit(empty(s));                         // the stage is free once these MMAs are done
                     if (kc == n_kc - 1) ptx::tc_commit(acc_full(u));  // and so is the pair's accumulator
@@ -191,15 +198,15 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_co
             if (ok) ok = ptx::mbar_wait(acc_full(u), (q >> 1) & 1);
             __syncwarp();
             ptx::tc_fence_after();
-            const int row0 = (cta + q * n_cta) * 2 * R;
+            const int row0 = (cta + q * n_cta) * TILES * R;
 #pragma unroll 1
-            for (int t = 0; t < 2; ++t) {
+            for (int t = 0; t < TILES; ++t) {
                 const int r = warp * 32 + lane;
                 const int v = r < R ? row0 + t * R + r : p.V;          // this thread's vocabulary row (none past R)
 #pragma unroll 1
                 for (int c = 0; c < N / 32; ++c) {
                     uint32_t acc[32];
-                    ptx::tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + (u * 2 + t) * N + c * 32, acc);
+                    ptx::tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + (u * TILES + t) * N + c * 32, acc);
                     ptx::tmem_ld_wait();
                     unsigned long long key[32];
 #pragma unroll
@@ -263,13 +270,14 @@ extern "C" int lm_head_argmax(const mtv_tree_t *tree, int B, int H, int V, const
     if (H < 64 || H % 64 != 0) return MTV_ERR_UNSUPPORTED_SHAPE;
     if (((uintptr_t)x | (uintptr_t)W) & 15) return MTV_ERR_INVALID_ARG;
     const int M = B * tree->T;
-    const int N = M <= 64 ? 64 : 128;
+    const int N = M <= 64 ? 64 : M <= 128 ? 128 : 256;
+    const int tiles = N <= 128 ? 2 : 1;                  // weight tiles per stage (see the kernel)
     const int passes = (M + N - 1) / N;
-        cudaStream_t st = (cudaStream_t)stream;
+    cudaStream_t st = (cudaStream_t)stream;
     CUtensorMap w_map, x_map;
     LmParams p;
     p.keys = keys; p.dev_error = tree->d_error; p.M = M; p.H = H; p.V = V; p.N = N;
-    p.stage_bytes = LM_W_BYTES + N * 128;
+    p.stage_bytes = tiles * LM_TILE_BYTES + N * 128;
     p.n_stages = (int)((LM_SMEM_MAX - 1024) / p.stage_bytes);
     if (p.n_stages > LM_MAX_STAGES) p.n_stages = LM_MAX_STAGES;
     const size_t smem = 1024 + (size_t)p.n_stages * p.stage_bytes;
@@ -277,21 +285,23 @@ extern "C" int lm_head_argmax(const mtv_tree_t *tree, int B, int H, int V, const
     if (!attr_done) {
         MTV_CUDA_CHECK(cudaFuncSetAttribute(lm_head_argmax_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, LM_SMEM_MAX));
         MTV_CUDA_CHECK(cudaFuncSetAttribute(lm_head_argmax_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, LM_SMEM_MAX));
+        MTV_CUDA_CHECK(cudaFuncSetAttribute(lm_head_argmax_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, LM_SMEM_MAX));
         attr_done = true;
     }
     MTV_CUDA_CHECK(cudaMemsetAsync(keys, 0, (size_t)M * 8, st));
     int ctas = sm_count() / passes;                      // per pass; one CTA per SM in all
-    const int min_pairs = (V + 255) / 256;
+    const int min_pairs = (V + tiles * 128 - 1) / (tiles * 128);   // units of `tiles` weight tiles
     if (ctas > (V + 63) / 64) ctas = (V + 63) / 64;      // no tile below 32 rows
     if (ctas < 1) ctas = 1;
     // every CTA walks the same number of tile pairs; the tile height shrinks until they just cover V
     const int rounds = (min_pairs + ctas - 1) / ctas;
     p.n_pairs = ctas * rounds;
-    p.R = ((V + 2 * p.n_pairs - 1) / (2 * p.n_pairs) + 7) / 8 * 8;
+    p.R = ((V + tiles * p.n_pairs - 1) / (tiles * p.n_pairs) + 7) / 8 * 8;
     if (!tma_map_2d_bf16(&w_map, W, V, H, p.R) || !tma_map_2d_bf16(&x_map, x, M, H, N)) return MTV_ERR_CUDA;
     const dim3 grid(passes, ctas);
     if (N == 64) lm_head_argmax_kernel<64><<<grid, LM_THREADS, smem, st>>>(w_map, x_map, p);
-    else lm_head_argmax_kernel<128><<<grid, LM_THREADS, smem, st>>>(w_map, x_map, p);
+    else if (N == 128) lm_head_argmax_kernel<128><<<grid, LM_THREADS, smem, st>>>(w_map, x_map, p);
+    else lm_head_argmax_kernel<256><<<grid, LM_THREADS, smem, st>>>(w_map, x_map, p);
     if (am) lm_head_finish_kernel<<<(M + 127) / 128, 128, 0, st>>>(M, keys, am, am_val);
     MTV_CUDA_CHECK(cudaGetLastError());
     return MTV_OK;

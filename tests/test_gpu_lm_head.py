@@ -48,6 +48,8 @@ LM_CASES = [
     (5, ("rank_prior", 4, (), 64), 128, 777),              # 320 nodes: three passes, the last one partial
     (3, ("cartesian", 1, (2,), 0), 64, 50),                # fewer vocabulary rows than one tile
     (1, ("rank_prior", 5, (), 128), 1024, 40000),          # more tile pairs than SMs
+    (3, ("rank_prior", 4, (), 64), 256, 3001),             # 192 nodes: one partial pass of 256
+    (9, ("rank_prior", 4, (), 64), 128, 20000),            # 576 nodes: three passes of 256, the last one partial
 ]
 
 
