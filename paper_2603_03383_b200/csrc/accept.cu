@@ -3,6 +3,8 @@
 // gather of the accepted tokens through retrieve_indices — all on the device.
 #include <cstdio>
 
+#include <cuda_bf16.h>
+
 #include "common.cuh"
 
 namespace mtv {
@@ -46,8 +48,12 @@ node_argmax_partial_kernel(int V, const __nv_bfloat16 *__restrict__ logits, unsi
     unsigned long long best = 0;
     const bool aligned = (((size_t)row * V) % 8) == 0;
     if (aligned) {
-        // four independent 16-byte loads in flight per thread, then the (cheap) key arithmetic
+        // Four independent 16-byte loads in flight per thread.  Per chunk of 8 logits only its maximum is formed
+        // (packed bf16 max) and compared with the thread's running maximum; the chunk that first raised it is
+        // looked at again at the end to find the element, so the scan costs about one instruction per logit.
         constexpr int U = 4;
+        float smax = -INFINITY;
+        int pos = -1;                      // first element of the chunk that holds the thread's maximum so far
         for (int i0 = begin + threadIdx.x * 8; i0 < end; i0 += U * ARGMAX_THREADS * 8) {
             uint4 u[U];
 #pragma unroll
@@ -62,16 +68,21 @@ node_argmax_partial_kernel(int V, const __nv_bfloat16 *__restrict__ logits, unsi
             for (int k = 0; k < U; ++k) {
                 const int i = i0 + k * ARGMAX_THREADS * 8;
                 if (i + 8 <= end) {
-                    const uint32_t w[4] = {u[k].x, u[k].y, u[k].z, u[k].w};
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        best = umax64(best, pack_key(w[j] & 0xffffu, i + 2 * j));
-                        best = umax64(best, pack_key(w[j] >> 16, i + 2 * j + 1));
-                    }
+                    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u[k]);
+                    const __nv_bfloat162 m2 = __hmax2(__hmax2(h[0], h[1]), __hmax2(h[2], h[3]));
+                    const float m = fmaxf(__low2float(m2), __high2float(m2));
+                    if (pos < 0 || m > smax) { smax = m; pos = i; }     // strictly greater: the first chunk stays
                 } else if (i < end) {
                     for (int j = i; j < end; ++j) best = umax64(best, pack_key(p[j], j));
                 }
             }
+        }
+        if (pos >= 0) {
+            // the first element of that chunk that equals the maximum (-0.0 == +0.0, as in the key)
+            int j = 0;
+            while (j < 7 && !(__uint_as_float((uint32_t)p[pos + j] << 16) == smax)) ++j;
+            if (!(__uint_as_float((uint32_t)p[pos + j] << 16) == smax)) j = 0;   // a chunk of NaNs
+            best = umax64(best, pack_key(p[pos + j], pos + j));
         }
     } else {
         for (int i = begin + threadIdx.x; i < end; i += ARGMAX_THREADS) best = umax64(best, pack_key(p[i], i));
