@@ -76,7 +76,7 @@ static_assert(TC_WBUF_OFF + TC_WBUF_ENTRIES * 8 <= TC_TILES_BYTES, "merge buffer
 static_assert((256 + TC_MAX_SPLITS) * TC_ROW_BYTES <= TC_PARK_ML_OFF, "rows to merge must fit below the small buffers");
 
 // barrier slots (8 bytes each) inside the barrier region
-enum { BAR_Q = 0, BAR_KV_FULL = 1, BAR_KV_EMPTY = BAR_KV_FULL + TC_SLOTS, BAR_S = BAR_KV_EMPTY + TC_SLOTS,
+enum { BAR_Q = 0 /* one per row tile */, BAR_KV_FULL = 2, BAR_KV_EMPTY = BAR_KV_FULL + TC_SLOTS, BAR_S = BAR_KV_EMPTY + TC_SLOTS,
        BAR_P = BAR_S + 2, BAR_O = BAR_P + 2, BAR_FINAL = BAR_O + 2, BAR_MERGE = BAR_FINAL + 1, BAR_COUNT = BAR_MERGE + 1 };
 static_assert(BAR_COUNT * 8 + 8 <= TC_BAR_BYTES, "barrier region too small");
 
@@ -177,6 +177,7 @@ __device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
         if (!SOFTMAX) {
             if (warp == TC_TMA_WARP && lane == 0) {
                 ptx::mbar_wait(bar(BAR_Q), 0);
+                if (c.nt == 2) ptx::mbar_wait(bar(BAR_Q + 1), 0);
                 for (int s = 0; s < TC_SLOTS; ++s) { ptx::mbar_wait(bar(BAR_KV_FULL + s), 0); ptx::mbar_wait(bar(BAR_KV_FULL + s), 1); }
             }
             if (warp == TC_MMA_WARP) {
@@ -324,6 +325,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
 
     if (warp == TC_TMA_WARP && lane == 0) {
         ptx::mbar_init(bar(BAR_Q), 1);
+        ptx::mbar_init(bar(BAR_Q + 1), 1);
+        // the copy engine fetches the three descriptors while the CTA sets itself up (they are kernel parameters:
+        // nothing the previous kernel of the stream could still be writing)
+        ptx::prefetch_tensormap(&k_map);
+        ptx::prefetch_tensormap(&q_map);
+        ptx::prefetch_tensormap(&v_map);
         for (int s = 0; s < TC_SLOTS; ++s) { ptx::mbar_init(bar(BAR_KV_FULL + s), 1); ptx::mbar_init(bar(BAR_KV_EMPTY + s), 1); }
         for (int t = 0; t < 2; ++t) {
             ptx::mbar_init(bar(BAR_S + t), 1);
@@ -377,13 +384,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
 
     if (warp == TC_TMA_WARP && lane == 0) {
         if (cnt > 0) {
-            // first K tile, then Q, then the rest: the first MMA needs K_0 and Q
+            // first K tile, then Q (a barrier per row tile: the first MMA needs K_0 and the first tile only), then the rest
             issue_kv(0);
-            ptx::mbar_arrive_expect_tx(bar(BAR_Q), nt * TC_TILE_BYTES);
-            for (int t = 0; t < nt; ++t)
+            for (int t = 0; t < nt; ++t) {
+                ptx::mbar_arrive_expect_tx(bar(BAR_Q + t), TC_TILE_BYTES);
                 for (int half = 0; half < 2; ++half)
-                    ptx::tma_load_4d(q_smem + t * TC_TILE_BYTES + half * TC_HALF_BYTES, &q_map, bar(BAR_Q), half * 64,
+                    ptx::tma_load_4d(q_smem + t * TC_TILE_BYTES + half * TC_HALF_BYTES, &q_map, bar(BAR_Q + t), half * 64,
                                      g * p.G, (rows0 + t * 128) / p.G, b);
+            }
             for (int i = 1; i < n_early; ++i) issue_kv(i);
         }
     }
@@ -431,6 +439,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
                 if (lane == 0) {
                     issue_S(0, 0);
                     ptx::tc_commit(bar(BAR_S + 0));
+                }
+                __syncwarp();
+                if (nt == 2) ok = ptx::mbar_wait(bar(BAR_Q + 1), 0);
+                ptx::tc_fence_after();
+                if (ok && lane == 0) {
                     if (nt == 2) { issue_S(1, 0); ptx::tc_commit(bar(BAR_S + 1)); }
                     ptx::tc_commit(bar(BAR_KV_EMPTY + 0));
                 }
