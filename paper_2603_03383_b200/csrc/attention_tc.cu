@@ -380,7 +380,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
                              (t_begin + i / 2) * TC_BN, g, b);
     };
     const int n_loads = 2 * cnt;
-    const int n_early = min(n_loads, TC_SLOTS);   // loads that need no free slot: issued before the CTA syncs
+    // Only the first K and V tiles are requested before the CTA syncs; the others wait until the first query tile
+    // has landed, so that what the first MMAs need is not queued behind 160 KB of tiles that are needed later.
+    const int n_early = min(n_loads, 2);
 
     if (warp == TC_TMA_WARP && lane == 0) {
         if (cnt > 0) {
@@ -407,9 +409,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
         reg_dec<TC_REGS_OTHER>();   // the whole fifth warpgroup gives registers to the softmax warpgroups
         if (warp == TC_TMA_WARP) {
             // ------------------------------------------------------------ TMA producer (the rest of the tiles)
+            if (cnt > 0 && !ptx::mbar_wait(bar(BAR_Q), 0)) *abort_flag = 1;
             for (int i = n_early; i < n_loads && !*abort_flag; ++i) {
                 const int slot = i % TC_SLOTS, use = i / TC_SLOTS;
-                if (!ptx::mbar_wait(bar(BAR_KV_EMPTY + slot), (use - 1) & 1)) { *abort_flag = 1; break; }
+                if (use > 0 && !ptx::mbar_wait(bar(BAR_KV_EMPTY + slot), (use - 1) & 1)) { *abort_flag = 1; break; }
                 if (lane == 0) issue_kv(i);
                 __syncwarp();
             }
