@@ -150,6 +150,7 @@ extern "C" int tree_accept(const mtv_tree_t *tree, int B, int V, const mtv_bf16 
         !acc_tok || !next_root || !ws || B < 1 || V < 1)
         return MTV_ERR_INVALID_ARG;
     if (tree->P > 255) return MTV_ERR_UNSUPPORTED_SHAPE;
+    if ((uintptr_t)logits & 15) return MTV_ERR_INVALID_ARG;   // the scan reads 16-byte chunks of the rows
     const AcceptWs L = accept_ws_layout(tree, B, V);
     if (ws_bytes < L.total) return MTV_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
@@ -222,6 +223,7 @@ extern "C" int tree_accept_static_scratch(const mtv_tree_t *tree, int B, int V, 
         !acc_tok || !next_root || B < 1 || V < 1)
         return MTV_ERR_INVALID_ARG;
     if (tree->P > 255) return MTV_ERR_UNSUPPORTED_SHAPE;
+    if ((uintptr_t)logits & 15) return MTV_ERR_INVALID_ARG;   // the scan reads 16-byte chunks of the rows
     const AcceptWs L = accept_ws_layout(tree, B, V);
     if (L.total > ACCEPT_STATIC_SCRATCH_BYTES) {
         char msg[160];

@@ -1,101 +1,116 @@
 // Tree attention on the 5th-generation tensor cores (Section 3.2 / Fig. 2(b)), head_dim 128.
 //
-// One CTA owns up to 256 query rows (two 128-row tiles of the (node, head-in-group) block
-// that shares one KV head) and a contiguous range of 128-key tiles.  Warp roles:
-//   warps 0-7 / 8-15 softmax warps of row tile 0 / 1: two threads per query row, each with one
-//                    half (64 keys) of the row of S from tensor memory in registers — two such warps
-//                    per scheduler, so that one can use the special-function unit while the other
-//                    issues the rest; they apply the ancestor bitmask on the tiles that overlap the
-//                    tree rows, agree on the running max through shared memory, keep partial row
-//                    sums and write P (bf16) back to tensor memory over S;
-//   warp 16          issues tcgen05.mma: S_t = Q_t K^T (operands in shared memory) and
-//                    O_t += P_t V (P from tensor memory, V from shared memory, N-major);
-//   warp 17          TMA producer: Q once, then K and V tiles through a ring of 32 KB slots;
-//   warps 18-19      only help with the copies of the merge.
-// Tensor memory: S0 | S1 | O0 | O1, 128 fp32 columns each; P_t overlays the first 64 columns
-// of S_t.  The softmax warpgroups take registers from the fifth warpgroup (setmaxnreg).
+// A pair of CTAs (a cluster of two) owns up to 256 query rows — the (node, head-in-group) rows that
+// share one KV head — and every nsplit-th 128-key group of the sequence.  The two CTAs form one
+// tcgen05 CTA pair: each keeps 128 of the query rows, its own S / P / O in tensor memory and its own
+// softmax warps, and each loads HALF of every K and V group from global memory (K: 64 of the 128 keys;
+// V: 64 of the 128 columns), so a K/V byte crosses from L2 to the SMs once per 256 query rows.  The
+// MMAs (M = 256 over the pair, N = 128) are issued by two threads of the even-ranked CTA and read both halves.
 //
-// The key splits of one query block are merged inside the same launch.  After its last key tile
-// a CTA parks its partial in shared memory — its own normalised result O / l in bf16 plus the
-// fp32 pair (m, l); the exchange of partials is bound by L2 bandwidth, so they travel in the
-// output's precision — sends it to the workspace with bulk copies (it stays in L2), and arrives
-// on a counter of its query block.  When all splits of
-// the block have arrived, every CTA fetches a slice of the rows of all partials with bulk copies
-// (plain loads would be throttled by the little L1 this kernel leaves), combines them in fp32 with
-// the weights exp2(m_s - m) l_s / sum and writes bf16 output rows.  The grid never exceeds one CTA per SM, so all CTAs are resident together and
-// the wait on the counter always ends; it is bounded all the same.  The counters live in the
-// tree object, start at zero and are put back to zero by the last CTA that has seen them full.
+// The two 64-key halves of a group belong to two STREAMS, each with its own accumulator O and its own
+// running (max, sum) per row; the streams are merged in registers at the end.  One softmax thread owns one
+// query row of one stream: it reads the 64 scores of its half from tensor memory, needs nobody else for the
+// row maximum, and writes P (bf16) back over them.  Every scheduler therefore runs two independent softmax
+// warps (one per stream): while one uses the special-function unit for its exponentials, the other waits
+// for tensor memory, barriers or the tensor core — the latencies that dominate a tile when all warps of a
+// scheduler move in lockstep.
+// Warp roles in each CTA:
+//   warps 0-3 / 4-7  softmax warps of stream 0 / 1 (warp w: tensor-memory lanes 32 (w % 4) ..);
+//   warp 8           (even CTA only) issues S = Q K^T of a whole group (operands in shared memory);
+//   warp 9           TMA producer of this CTA's halves: Q once, K and V through rings of 16 KB slots;
+//   warp 10          relay: tells the issuing CTA when this CTA's half of a group has landed (after clearing
+//                    V rows past the last key);
+//   warp 11          (even CTA only) issues O += P V per stream (P from tensor memory, V N-major from
+//                    shared memory).
+// Tensor memory per CTA: two S buffers of 128 columns (64 per stream; P overlays the first 32 columns of a
+// stream's 64), then O of stream 0 and O of stream 1 (128 columns each).  S of group i + 2 is issued as soon as
+// both O += P V of group i have completed, two groups ahead of the softmax.  Ring slots are handed back to the
+// producer by the softmax warps, which see S of group i complete (its K slot is free) and with it O += P V
+// of group i - 2 (its V slot is free): no tensor-core commit is spent on it.
 //
-// The running max is only raised when the new row max exceeds it by more than 8 (in log2
-// units), so O in tensor memory is rescaled rarely; P stays below 2^8.
+// The key splits of a query block are merged inside the launch.  After its last group a CTA writes its own
+// normalised result O / l (bf16) and (m, l) to the workspace, one thread release-arrives on a counter of the
+// (query block, CTA rank), and when all splits have arrived each CTA combines a slice of the rows:
+// out = sum_s w_s (O_s / l_s) with w_s = exp2(m_s - m) l_s / sum.  This wait needs all CTAs of a query
+// block resident together: splits are only planned when the whole grid fits the device in one wave (one CTA
+// per SM); the wait is bounded all the same.  Without splits CTAs never wait for CTAs outside their pair
+// and the grid may be of any size.
+//
+// The running max of a stream moves only when a tile's max exceeds it by more than 8 (log2 units), so O is
+// rescaled rarely and P stays below 2^8.
+//
+// Build option -DMTV_TRACE: per-CTA cycle stamps of the phases through mtv_trace_set (development aid).
 #include <cuda.h>
+
+#include <type_traits>
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
 namespace mtv {
 
-constexpr int TC_BN = 128;
-constexpr int TC_SLOTS = 5;
-constexpr int TC_THREADS = 640;   // 5 warpgroups: 4 of softmax warps, {MMA warp, TMA warp, 2 helper warps}
-constexpr int TC_MMA_WARP = 16, TC_TMA_WARP = 17;
-constexpr uint32_t TC_TILE_BYTES = 128 * 128 * 2;   // one 128 x 128 bf16 tile: two 64-column halves
-constexpr uint32_t TC_HALF_BYTES = TC_TILE_BYTES / 2;
-constexpr uint32_t TC_Q_BYTES = 2 * TC_TILE_BYTES;
-constexpr uint32_t TC_RING_BYTES = TC_SLOTS * TC_TILE_BYTES;
-constexpr uint32_t TC_BAR_BYTES = 256;
-constexpr uint32_t TC_XMAX_BYTES = 2 * 2 * 128 * 2;   // running-max exchange of the two half-row threads, bf16
-constexpr uint32_t TC_SMEM_BYTES = 1024 + TC_Q_BYTES + TC_RING_BYTES + TC_BAR_BYTES + TC_XMAX_BYTES;
+constexpr int TC_BN = 128;        // keys per group of a CTA pair (one S MMA set); a stream takes 64 of them
+constexpr int TC_HALF = TC_BN / 2;
+constexpr int TC_STAGES = 5;      // K and V ring slots per CTA
+constexpr int TC_THREADS = 384;
+constexpr int TC_SOFTMAX_WARPS = 8;
+constexpr int TC_MMA_WARP = 8, TC_TMA_WARP = 9, TC_RELAY_WARP = 10, TC_PV_WARP = 11;
+constexpr uint32_t TC_Q_BYTES = 128 * 128 * 2;   // this CTA's 128 query rows: two 64-column halves
+constexpr uint32_t TC_Q_HALF = TC_Q_BYTES / 2;
+constexpr uint32_t TC_K_BYTES = 64 * 128 * 2;    // this CTA's 64 keys of a group: two 64-column halves
+constexpr uint32_t TC_K_HALF = TC_K_BYTES / 2;
+constexpr uint32_t TC_V_BYTES = 128 * 64 * 2;    // 128 keys x this CTA's 64 columns
+constexpr uint32_t TC_BAR_BYTES = 1024;
+constexpr uint32_t TC_ML_BYTES = 2 * 128 * 8;    // (m, l) per stream and row, for the merge of the two streams
+constexpr uint32_t TC_OFF_K = TC_Q_BYTES;
+constexpr uint32_t TC_OFF_V = TC_OFF_K + TC_STAGES * TC_K_BYTES;
+constexpr uint32_t TC_OFF_BAR = TC_OFF_V + TC_STAGES * TC_V_BYTES;
+constexpr uint32_t TC_OFF_ML = TC_OFF_BAR + TC_BAR_BYTES;
+constexpr uint32_t TC_SMEM_BYTES = 1024 + TC_OFF_ML + TC_ML_BYTES;
 static_assert(TC_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 constexpr float TC_RESCALE_THRESHOLD = 8.f;
 constexpr int TC_MAX_SPLITS = 32;
-constexpr int TC_MAX_GROUPS = 256;   // merge counters available in the tree object
+constexpr int TC_MAX_COUNTERS = 256;   // merge counters in the tree object: one per (query block, CTA rank)
 
-// Register rebalancing.  The CTA's pool is what the launch allocates: TC_THREADS threads at the
-// per-thread count the compiler derives from the launch bounds (65536 / 640 rounded down to a
-// multiple of 8 = 96).  setmaxnreg.inc blocks until the pool has the registers, so the five
-// warpgroups' targets must not add up to more than the pool: 4 x 104 + 64 = 5 x 96.
-constexpr int TC_REGS_LAUNCH = 96, TC_REGS_SOFTMAX = 104, TC_REGS_OTHER = 64;
-static_assert(4 * TC_REGS_SOFTMAX + TC_REGS_OTHER <= 5 * TC_REGS_LAUNCH, "setmaxnreg targets exceed the CTA's register pool");
-static_assert(TC_REGS_LAUNCH * TC_THREADS <= 65536, "launch register count does not fit the register file");
+// tensor-memory columns: S buffer b of stream t at 128 b + 64 t (P over its first 32 columns), O of stream t at 256 + 128 t
+constexpr uint32_t TM_S = 0, TM_O = 256;
 
-// After the last key tile the Q / K / V buffers are reused:
-//   [0, 64 KB)       the parked partial: 256 rows of 128 bf16 values O / l (the split's own normalised
-//                    result; fp32 (m, l) travel beside it).  16-byte chunk j of row r sits at chunk
-//                    position j ^ (r & 15): the one-row-per-thread stores are conflict-free while rows
-//                    stay contiguous for one bulk copy.  The workspace holds partials in the same
-//                    form; whoever reads a row undoes the permutation.  After the partial has left
-//                    for the workspace the same space receives the rows this CTA merges.
-//   the last 8 KB    parked (m, l) per row; (m, l) then the merge weights of every split
-constexpr uint32_t TC_ROW_BYTES = 256;
-constexpr uint32_t TC_TILES_BYTES = TC_Q_BYTES + TC_RING_BYTES;
-constexpr uint32_t TC_PARK_ML_OFF = TC_TILES_BYTES - 8192;
-constexpr uint32_t TC_WBUF_OFF = TC_PARK_ML_OFF + 256 * 8;
-constexpr uint32_t TC_WBUF_ENTRIES = 256 + TC_MAX_SPLITS;
-static_assert(TC_WBUF_OFF + TC_WBUF_ENTRIES * 8 <= TC_TILES_BYTES, "merge buffers must fit the tile buffers");
-static_assert((256 + TC_MAX_SPLITS) * TC_ROW_BYTES <= TC_PARK_ML_OFF, "rows to merge must fit below the small buffers");
+// mbarrier slots (8 bytes each).  "ready", "sfree" and "pready" are only used in the issuing CTA.
+enum {
+    BAR_QFULL = 0,
+    BAR_KFULL = 1,
+    BAR_VFULL = BAR_KFULL + TC_STAGES,
+    BAR_KFREE = BAR_VFULL + TC_STAGES,
+    BAR_VFREE = BAR_KFREE + TC_STAGES,
+    BAR_QREADY = BAR_VFREE + TC_STAGES,
+    BAR_KREADY = BAR_QREADY + 1,
+    BAR_VREADY = BAR_KREADY + TC_STAGES,
+    BAR_SREADY = BAR_VREADY + TC_STAGES,   // [2 buffers] S of a group is complete (tensor core -> softmax warps of both CTAs)
+    // Barriers whose phases follow the groups come in pairs (even and odd groups): a waiter may then lag at most one
+    // phase behind, which is all a parity wait can tell apart.
+    BAR_PREADY = BAR_SREADY + 2,           // [2] both streams' P are in tensor memory (softmax warps of both CTAs -> issuer)
+    BAR_ODONE = BAR_PREADY + 2,            // [2] both streams' O += P V of a group are complete (tensor core -> both CTAs)
+    BAR_FINAL = BAR_ODONE + 2,
+    BAR_COUNT = BAR_FINAL + 1
+};
+static_assert(BAR_COUNT * 8 + 16 <= TC_BAR_BYTES, "barrier region too small");
 
-// barrier slots (8 bytes each) inside the barrier region
-enum { BAR_Q = 0 /* one per row tile */, BAR_KV_FULL = 2, BAR_KV_EMPTY = BAR_KV_FULL + TC_SLOTS, BAR_S = BAR_KV_EMPTY + TC_SLOTS,
-       BAR_P = BAR_S + 2, BAR_O = BAR_P + 2, BAR_FINAL = BAR_O + 2, BAR_MERGE = BAR_FINAL + 1, BAR_COUNT = BAR_MERGE + 1 };
-static_assert(BAR_COUNT * 8 + 8 <= TC_BAR_BYTES, "barrier region too small");
-
-// instruction descriptors: bf16 x bf16 -> fp32, M = 128, N = 128
-constexpr uint32_t IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr uint32_t IDESC_QK = IDESC_BASE;               // A, B both K-major
-constexpr uint32_t IDESC_PV = IDESC_BASE | (1u << 16);  // B (= V) N-major
+// instruction descriptors: bf16 x bf16 -> fp32, M = 256 over the CTA pair
+constexpr uint32_t IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 4) << 24);
+constexpr uint32_t IDESC_QK = IDESC_BASE | ((128u >> 3) << 17);                // N = 128 keys; A, B both K-major
+constexpr uint32_t IDESC_PV = IDESC_BASE | ((128u >> 3) << 17) | (1u << 16);   // N = 128 columns; B (= V) N-major
 
 struct TcParams {
     const int32_t *seq_lens;
     const uint64_t *anc;   // [T][2]
     __nv_bfloat16 *out;    // [B][T][Hq][128]
-    __nv_bfloat16 *ws_o;   // [groups][nsplit][256 rows][128] partial O / l, chunks permuted (only when nsplit > 1)
-    float2 *ws_ml;         // [groups][nsplit][256] partial (m, l)
-    int32_t *arrive, *depart;   // [groups] merge counters, zero between calls
+    __nv_bfloat16 *ws_o;   // [query blocks][nsplit][256 rows][128] partial O / l (only when nsplit > 1)
+    float2 *ws_ml;         // [query blocks][nsplit][256] partial (m, l)
+    int32_t *arrive, *depart;   // [query blocks][2] merge counters, zero between calls
     int32_t *status;       // [B] or null
     int32_t *dev_error;
     float scale_log2;
-    int T, G, Hq, Hkv, Lcap, nsplit, n_rt, M_rows;
+    int T, G, Hq, Hkv, Lcap, nsplit, n_blk, M_rows;
 };
 
 // 128-byte-swizzled shared-memory operand descriptor.
@@ -109,16 +124,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes
 }
 // K-major operand (rows 128 bytes apart inside an 8-row group, groups 1024 bytes apart)
 __device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr) { return smem_desc(saddr, 16, 1024); }
-// N-major operand: 64-column halves TC_HALF_BYTES apart, 8-key groups 1024 bytes apart
-__device__ __forceinline__ uint64_t desc_nmajor(uint32_t saddr) { return smem_desc(saddr, TC_HALF_BYTES, 1024); }
+// N-major operand one 64-column swizzle atom wide: 8-key groups 1024 bytes apart
+__device__ __forceinline__ uint64_t desc_nmajor(uint32_t saddr) { return smem_desc(saddr, TC_V_BYTES, 1024); }
 
-// Register rebalancing between warpgroups (all four warps of a warpgroup execute it).
-template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
-template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
-
-// CTA-wide barrier usable from the diverged warp roles (every thread of the CTA arrives on it,
-// from whichever copy of the epilogue it runs).
 __device__ __forceinline__ void cta_sync() { asm volatile("bar.sync 1, %0;" ::"n"(TC_THREADS) : "memory"); }
+__device__ __forceinline__ void softmax_sync() { asm volatile("bar.sync 6, %0;" ::"n"(TC_SOFTMAX_WARPS * 32) : "memory"); }
 
 __device__ __forceinline__ float ex2(float x) {
     float y;
@@ -136,536 +146,572 @@ __device__ __forceinline__ int ld_acquire(const int32_t *p) {
     return v;
 }
 
-// Developer timeline (compiled out unless MTV_TRACE is defined): lane 0 of the calling warp
-// stores the SM cycle counter of event `id` for this CTA.
 #ifdef MTV_TRACE
 __device__ long long *g_trace = nullptr;   // [ctas][64]
-#define TRACE_CTA ((size_t)(blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x)
-#define TRACE(id)                                                                      \
-    do {                                                                               \
-        if (g_trace && (threadIdx.x % 32) == 0) g_trace[TRACE_CTA * 64 + (id)] = clock64(); \
+// the buffer's address is read once per thread (TRACE_INIT); a stamp is then one clock read and one store
+#define TRACE_INIT                                                                                                  \
+    long long *trace_row = g_trace;                                                                                 \
+    if (trace_row) trace_row += ((size_t)(blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * 64
+#define TRACE(id)                                                            \
+    do {                                                                     \
+        if (trace_row && (threadIdx.x % 32) == 0) trace_row[(id)] = clock64(); \
     } while (0)
 #else
+#define TRACE_INIT
 #define TRACE(id)
 #endif
 
-// What the epilogue needs from the main body.
-struct TcCtx {
-    unsigned char *tiles;   // 1024-byte aligned base of the tile buffers (generic address)
-    uint32_t bars;          // shared address of the barrier region
-    volatile int *abort_flag;
-    uint32_t tmem;
-    int nt, split, rows0, g, b, cnt;
-    bool final_committed;
-};
-
-// Everything after the last key tile; instantiated once for the softmax warpgroups (which have
-// the registers to keep many loads in flight) and once for the third warpgroup.
-template <bool SOFTMAX>
-__device__ __forceinline__ void tc_epilogue(const TcParams &p, const TcCtx &c) {
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    float2 *wbuf = reinterpret_cast<float2 *>(c.tiles + TC_WBUF_OFF);
-    auto bar = [&](int i) { return c.bars + (uint32_t)i * 8u; };
-
-    ptx::tc_fence_before();
-    cta_sync();   // every role is done; partials are parked
-    if (*c.abort_flag) {
-        // A bounded wait ran out: raise the sticky error, give outstanding copies and tensor-core
-        // work one more bounded chance to finish.  The CTA still takes part in the merge so that
-        // the other splits never wait for it; the error word tells the host the output is invalid.
-        if (threadIdx.x == 0) atomicExch(p.dev_error, MTV_ERR_TIMEOUT);
-        if (!SOFTMAX) {
-            if (warp == TC_TMA_WARP && lane == 0) {
-                ptx::mbar_wait(bar(BAR_Q), 0);
-                if (c.nt == 2) ptx::mbar_wait(bar(BAR_Q + 1), 0);
-                for (int s = 0; s < TC_SLOTS; ++s) { ptx::mbar_wait(bar(BAR_KV_FULL + s), 0); ptx::mbar_wait(bar(BAR_KV_FULL + s), 1); }
-            }
-            if (warp == TC_MMA_WARP) {
-                if (!c.final_committed && lane == 0) ptx::tc_commit(bar(BAR_FINAL));
-                __syncwarp();
-                ptx::mbar_wait(bar(BAR_FINAL), 0);
-            }
-        }
-        cta_sync();
-    }
-    if (warp == 0) TRACE(44);   // partial parked
-
-    const int act_rows = c.nt * 128;
-    const int nsplit = p.nsplit;
-    const int grp = blockIdx.z * gridDim.y + blockIdx.y;
-    const unsigned char *rows_smem = c.tiles;   // parked rows, later the rows to merge
-    // chunk j (8 bf16 values) of a 256-byte row whose index inside its 256-row slab is r
-    auto chunk = [&](const unsigned char *row_ptr, int r, int j) {
-        return *reinterpret_cast<const uint4 *>(row_ptr + ((j ^ (r & 15)) << 4));
-    };
-    auto out_ptr = [&](int r, int j) {   // 8 output values of query-block row r
-        const int node = r / p.G, hq = c.g * p.G + r % p.G;
-        return reinterpret_cast<uint4 *>(p.out + (((size_t)c.b * p.T + node) * p.Hq + hq) * 128 + j * 8);
-    };
-    if (nsplit == 1) {
-        // the parked partial is the result
-        for (int item = threadIdx.x; item < act_rows * 16; item += TC_THREADS) {
-            const int row = item / 16, j = item % 16, r = c.rows0 + row;
-            if (r < p.M_rows) *out_ptr(r, j) = chunk(rows_smem + row * TC_ROW_BYTES, row, j);
-        }
-    } else {
-        const size_t slab0 = (size_t)grp * nsplit;   // first slab of this query block
-        const int rows_per = (act_rows + nsplit - 1) / nsplit;
-        const int row_begin = c.split * rows_per;
-        const int n_my = max(0, min(act_rows, row_begin + rows_per) - row_begin);
-        if (threadIdx.x == 0) {
-            // ---- publish: two bulk copies out of shared memory, then arrive and wait for the others
-            const size_t slab = slab0 + c.split;
-            ptx::bulk_s2g(p.ws_o + slab * 256 * 128, ptx::smem_u32(c.tiles), act_rows * TC_ROW_BYTES);
-            ptx::bulk_s2g(p.ws_ml + slab * 256, ptx::smem_u32(c.tiles + TC_PARK_ML_OFF), act_rows * 8);
-            ptx::bulk_commit();
-            ptx::bulk_wait_all();
-            TRACE(51);   // partial left shared memory and is written
-            ptx::fence_proxy_async_global();
-            // release-arrive without waiting for the counter's old value
-            asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(p.arrive + grp) : "memory");
-            TRACE(52);   // arrived
-            const long long t0 = clock64();
-            while (ld_acquire(p.arrive + grp) < nsplit)
-                if (clock64() - t0 > ptx::WAIT_CYCLE_LIMIT) { atomicExch(p.dev_error, MTV_ERR_TIMEOUT); break; }
-            TRACE(53);   // everybody arrived
-        }
-        cta_sync();
-        // ---- fetch rows [row_begin, row_begin + n_my) of every split: one bulk copy per split, each issued by a
-        //      different warp (the copies of one warp's lanes are issued one after the other)
-        if (n_my > 0 && lane == 0) {
-            if (warp == 0) ptx::mbar_arrive_expect_tx(bar(BAR_MERGE), (uint32_t)(nsplit * n_my) * TC_ROW_BYTES);
-            ptx::fence_proxy_async_global();   // the other CTAs' partials, acquired above, before the async-proxy reads
-            for (int sp = warp; sp < nsplit; sp += TC_THREADS / 32)
-                ptx::bulk_g2s(ptx::smem_u32(c.tiles) + (uint32_t)(sp * n_my) * TC_ROW_BYTES,
-                              p.ws_o + ((slab0 + sp) * 256 + row_begin) * 128, (uint32_t)n_my * TC_ROW_BYTES, bar(BAR_MERGE));
-        }
-        if (warp == 0) TRACE(45);   // all splits arrived, rows on their way
-        // Nobody polls the arrival counter once all have seen it full: the last one to get here puts both counters
-        // back to zero (the next call cannot start before this kernel has ended).  Done here, behind the copies,
-        // so that the round trip of the atomic is not on the way of anything.
-        if (threadIdx.x == 0 && atomicAdd(p.depart + grp, 1) == nsplit - 1) {
-            p.arrive[grp] = 0;
-            p.depart[grp] = 0;
-            __threadfence();
-        }
-        // ---- merge weights, one warp per row, lane s = split s: exp2(m_s - m) l_s / sum over the splits
-        //      (split s contributes its own normalised result O_s / l_s)
-        for (int rl = warp; rl < n_my; rl += TC_THREADS / 32) {
-            float2 ml = make_float2(-INFINITY, 0.f);
-            if (lane < nsplit) ml = __ldcg(p.ws_ml + (slab0 + lane) * 256 + row_begin + rl);
-            float m = ml.x;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-            const float w = ml.x == -INFINITY ? 0.f : ex2(ml.x - m) * ml.y;
-            float lsum = w;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
-            if (lane < nsplit) wbuf[rl * nsplit + lane].x = w / lsum;
-        }
-        cta_sync();
-        if (warp == 0) TRACE(49);   // weights ready
-        if (n_my > 0 && !ptx::mbar_wait(bar(BAR_MERGE), 0) && threadIdx.x == 0) atomicExch(p.dev_error, MTV_ERR_TIMEOUT);
-        if (warp == 0) TRACE(50);   // rows landed
-        for (int item = threadIdx.x; item < n_my * 16; item += TC_THREADS) {
-            const int rl = item / 16, j = item % 16;
-            const int r = c.rows0 + row_begin + rl;
-            if (r >= p.M_rows) continue;
-            float acc[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-            const unsigned char *row_ptr = rows_smem + rl * TC_ROW_BYTES;
-#pragma unroll 6
-            for (int sp = 0; sp < nsplit; ++sp) {
-                const float w = wbuf[rl * nsplit + sp].x;
-                const uint4 v = chunk(row_ptr + (size_t)(sp * n_my) * TC_ROW_BYTES, row_begin + rl, j);
-                const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    acc[2 * e] = fmaf(w, __uint_as_float(vw[e] << 16), acc[2 * e]);
-                    acc[2 * e + 1] = fmaf(w, __uint_as_float(vw[e] & 0xffff0000u), acc[2 * e + 1]);
-                }
-            }
-            *out_ptr(r, j) = make_uint4(pack2_bf16(acc[0], acc[1]), pack2_bf16(acc[2], acc[3]),
-                                        pack2_bf16(acc[4], acc[5]), pack2_bf16(acc[6], acc[7]));
-        }
-        if (warp == 0) TRACE(46);   // merge done
-    }
-    if (!SOFTMAX && warp == TC_MMA_WARP) {
-        ptx::tc_fence_after();
-        ptx::tmem_dealloc(c.tmem, 512);
-    }
-    if (warp == 0) TRACE(47);
-}
-
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                     const __grid_constant__ CUtensorMap v_map, const TcParams p) {
     extern __shared__ unsigned char smem_raw[];
     // Programmatic dependent launch: let the next kernel of the stream be set up while this one runs.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int split = blockIdx.x;
-    const int g = blockIdx.y / p.n_rt, rt = blockIdx.y % p.n_rt;
+    const uint32_t rank = ptx::cluster_ctarank();     // 0: issues the MMAs, rows 0-127 of the block; 1: rows 128-255
+    const int split = blockIdx.x >> 1;
+    const int g = blockIdx.y / p.n_blk, blk = blockIdx.y % p.n_blk;
     const int b = blockIdx.z;
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    TRACE_INIT;
     if (warp == 0) TRACE(0);
 
-    // carve shared memory (tiles need 1024-byte alignment for the 128-byte swizzle)
+    // carve shared memory (tiles need 1024-byte alignment for the 128-byte swizzle); both CTAs of the pair
+    // get the same offsets, which the pair MMAs and the remote barrier addresses rely on
     const uint32_t raw = ptx::smem_u32(smem_raw);
     const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
-    const uint32_t q_smem = raw + pad;
-    const uint32_t ring = q_smem + TC_Q_BYTES;
-    const uint32_t bars = ring + TC_RING_BYTES;
-    unsigned char *tiles_gen = smem_raw + pad;
-    unsigned char *bar_region = tiles_gen + TC_Q_BYTES + TC_RING_BYTES;
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(bar_region + BAR_COUNT * 8);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bar_region + BAR_COUNT * 8 + 4);
+    const uint32_t sbase = raw + pad;
+    unsigned char *gbase = smem_raw + pad;
+    const uint32_t q_smem = sbase, k_ring = sbase + TC_OFF_K, v_ring = sbase + TC_OFF_V, bars = sbase + TC_OFF_BAR;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gbase + TC_OFF_BAR + BAR_COUNT * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(gbase + TC_OFF_BAR + BAR_COUNT * 8 + 4);
+    float2 *ml_x = reinterpret_cast<float2 *>(gbase + TC_OFF_ML);
     auto bar = [&](int i) { return bars + (uint32_t)i * 8u; };
-    float2 *park_ml = reinterpret_cast<float2 *>(tiles_gen + TC_PARK_ML_OFF);
+    auto lead = [&](int i) { return ptx::mapa(bar(i), 0); };        // the same barrier in the issuing CTA
+    auto peer = [&](int i) { return ptx::mapa(bar(i), rank ^ 1); }; // the same barrier in the other CTA
 
     if (warp == TC_TMA_WARP && lane == 0) {
-        ptx::mbar_init(bar(BAR_Q), 1);
-        ptx::mbar_init(bar(BAR_Q + 1), 1);
-        // the copy engine fetches the three descriptors while the CTA sets itself up (they are kernel parameters:
-        // nothing the previous kernel of the stream could still be writing)
         ptx::prefetch_tensormap(&k_map);
         ptx::prefetch_tensormap(&q_map);
         ptx::prefetch_tensormap(&v_map);
-        for (int s = 0; s < TC_SLOTS; ++s) { ptx::mbar_init(bar(BAR_KV_FULL + s), 1); ptx::mbar_init(bar(BAR_KV_EMPTY + s), 1); }
+        ptx::mbar_init(bar(BAR_QFULL), 1);
+        ptx::mbar_init(bar(BAR_QREADY), 2);
+        for (int s = 0; s < TC_STAGES; ++s) {
+            ptx::mbar_init(bar(BAR_KFULL + s), 1);
+            ptx::mbar_init(bar(BAR_VFULL + s), 1);
+            ptx::mbar_init(bar(BAR_KFREE + s), TC_SOFTMAX_WARPS);   // the softmax warps of this CTA
+            ptx::mbar_init(bar(BAR_VFREE + s), TC_SOFTMAX_WARPS);
+            ptx::mbar_init(bar(BAR_KREADY + s), 2);    // the relay warp of each CTA
+            ptx::mbar_init(bar(BAR_VREADY + s), 2);
+        }
         for (int t = 0; t < 2; ++t) {
-            ptx::mbar_init(bar(BAR_S + t), 1);
-            ptx::mbar_init(bar(BAR_P + t), 256);
-            ptx::mbar_init(bar(BAR_O + t), 1);
+            ptx::mbar_init(bar(BAR_SREADY + t), 1);
+            ptx::mbar_init(bar(BAR_PREADY + t), 2 * TC_SOFTMAX_WARPS);    // the softmax warps of both CTAs
+            ptx::mbar_init(bar(BAR_ODONE + t), 1);
         }
         ptx::mbar_init(bar(BAR_FINAL), 1);
-        ptx::mbar_init(bar(BAR_MERGE), 1);
         ptx::fence_mbar_init();
         *abort_flag = 0;
     }
     if (warp == TC_MMA_WARP) {
-        ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t *>(tmem_slot)), 512);
-        ptx::tmem_relinquish();
+        ptx::tmem_alloc_pair(ptx::smem_u32(const_cast<uint32_t *>(tmem_slot)), 512);
+        ptx::tmem_relinquish_pair();
     }
     ptx::tc_fence_before();
     __syncthreads();
+    // The peer's barriers and tensor memory must exist before anything is sent its way: a cluster barrier,
+    // whose wait comes after the sequence length has been read (both latencies overlap).
+    ptx::cluster_arrive();
     ptx::tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
     if (warp == 0) TRACE(1);
 
     // Nothing above touched global memory.  From here on the previous kernel of the stream must be
     // complete (its outputs may be this kernel's inputs, and it may share the workspace and counters).
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int L = p.seq_lens[b];
-    const bool reporter = blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0;
-    if (L + p.T > p.Lcap) {         // the same for every CTA of the query block: nobody waits for anybody
-        if (reporter && p.status) p.status[b] = MTV_ERR_CAPACITY;
-        if (warp == TC_MMA_WARP) ptx::tmem_dealloc(*tmem_slot, 512);
-        return;
+    const int rows0 = blk * 256 + (int)rank * 128;   // first row of this CTA inside the (sequence, KV head) block
+    auto tile_of = [&](int j) { return split + j * p.nsplit; };
+    auto issue_k = [&](int j) {
+        const int s = j % TC_STAGES;
+        ptx::mbar_arrive_expect_tx(bar(BAR_KFULL + s), TC_K_BYTES);
+        for (int half = 0; half < 2; ++half)
+            ptx::tma_load_4d(k_ring + s * TC_K_BYTES + half * TC_K_HALF, &k_map, bar(BAR_KFULL + s), half * 64,
+                             tile_of(j) * TC_BN + (int)rank * TC_HALF, g, b);
+    };
+    auto issue_v = [&](int j) {
+        const int s = j % TC_STAGES;
+        ptx::mbar_arrive_expect_tx(bar(BAR_VFULL + s), TC_V_BYTES);
+        ptx::tma_load_4d(v_ring + s * TC_V_BYTES, &v_map, bar(BAR_VFULL + s), (int)rank * 64, tile_of(j) * TC_BN, g, b);
+    };
+    constexpr int TC_EARLY = 2;   // tiles requested before the length is known
+    if (warp == TC_TMA_WARP && lane == 0) {
+        // The first tiles of this split and the query tile do not depend on the sequence length (the tiles of a split
+        // are split, split + nsplit, ...; past the end of the cache a copy delivers zeros), so they are requested while
+        // the length is still on its way; they only touch this CTA's own shared memory and barriers.
+        issue_k(0);
+        ptx::mbar_arrive_expect_tx(bar(BAR_QFULL), TC_Q_BYTES);
+        for (int half = 0; half < 2; ++half)
+            ptx::tma_load_4d(q_smem + half * TC_Q_HALF, &q_map, bar(BAR_QFULL), half * 64, g * p.G, rows0 / p.G, b);
+        issue_k(1);
+        issue_v(0);
+        issue_v(1);
     }
-    if (reporter && p.status) p.status[b] = MTV_OK;
+    const bool reporter = blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0;
+    const bool over = L + p.T > p.Lcap;   // the same for every CTA of the sequence: nobody waits for anybody
+    if (reporter && p.status) p.status[b] = over ? MTV_ERR_CAPACITY : MTV_OK;
     const int n_keys = L + p.T;
     const int tiles = (n_keys + TC_BN - 1) / TC_BN;
-    const int base_cnt = tiles / p.nsplit, rem = tiles % p.nsplit;
-    const int t_begin = split * base_cnt + min(split, rem);
-    const int cnt = base_cnt + (split < rem ? 1 : 0);
-    const int rows0 = rt * 256;
-    const int nt = p.M_rows - rows0 > 128 ? 2 : 1;
+    // key tiles split, split + nsplit, ... : the splits of a query block read neighbouring tiles at the same time
+    const int cnt = over || split >= tiles ? 0 : (tiles - split + p.nsplit - 1) / p.nsplit;
+    const bool have_rows = rows0 < p.M_rows;
+    if (warp != TC_TMA_WARP) ptx::cluster_wait();   // the producer first requests this CTA's own tiles
 
-    // One K or V tile into ring slot (i mod TC_SLOTS): i = 2j is K of key tile j, i = 2j + 1 is V.
-    auto issue_kv = [&](int i) {
-        const int slot = i % TC_SLOTS;
-        const CUtensorMap *map = (i & 1) ? &v_map : &k_map;
-        ptx::mbar_arrive_expect_tx(bar(BAR_KV_FULL + slot), TC_TILE_BYTES);
-        for (int half = 0; half < 2; ++half)
-            ptx::tma_load_4d(ring + slot * TC_TILE_BYTES + half * TC_HALF_BYTES, map, bar(BAR_KV_FULL + slot), half * 64,
-                             (t_begin + i / 2) * TC_BN, g, b);
+    // A wait that ran out: flag both CTAs of the pair and raise the sticky error.
+    auto give_up = [&]() {
+        *abort_flag = 1;
+        ptx::st_cluster_u32(ptx::mapa(ptx::smem_u32(const_cast<int *>(abort_flag)), rank ^ 1), 1u);
+        atomicExch(p.dev_error, MTV_ERR_TIMEOUT);
     };
-    const int n_loads = 2 * cnt;
-    // Only the first K and V tiles are requested before the CTA syncs; the others wait until the first query tile
-    // has landed, so that what the first MMAs need is not queued behind 160 KB of tiles that are needed later.
-    const int n_early = min(n_loads, 2);
 
-    if (warp == TC_TMA_WARP && lane == 0) {
-        if (cnt > 0) {
-            // first K tile, then Q (a barrier per row tile: the first MMA needs K_0 and the first tile only), then the rest
-            issue_kv(0);
-            for (int t = 0; t < nt; ++t) {
-                ptx::mbar_arrive_expect_tx(bar(BAR_Q + t), TC_TILE_BYTES);
-                for (int half = 0; half < 2; ++half)
-                    ptx::tma_load_4d(q_smem + t * TC_TILE_BYTES + half * TC_HALF_BYTES, &q_map, bar(BAR_Q + t), half * 64,
-                                     g * p.G, (rows0 + t * 128) / p.G, b);
+    if (warp == TC_TMA_WARP) {
+        // ------------------------------------------------------------ TMA producer: this CTA's halves
+        __syncwarp();
+        ptx::cluster_wait();
+        if (lane == 0) {
+            // tiles requested before the length was known and not needed after all: let them land before the CTA can exit
+            for (int j = cnt; j < TC_EARLY; ++j) {
+                ptx::mbar_wait(bar(BAR_KFULL + j), 0);
+                ptx::mbar_wait(bar(BAR_VFULL + j), 0);
             }
-            for (int i = 1; i < n_early; ++i) issue_kv(i);
+            if (cnt == 0) ptx::mbar_wait(bar(BAR_QFULL), 0);
         }
-    }
-    __syncwarp();
-
-    TcCtx ctx;
-    ctx.tiles = tiles_gen; ctx.bars = bars; ctx.abort_flag = abort_flag; ctx.tmem = *tmem_slot;
-    ctx.nt = nt; ctx.split = split; ctx.rows0 = rows0; ctx.g = g; ctx.b = b; ctx.cnt = cnt;
-    ctx.final_committed = false;
-    const uint32_t tmem = ctx.tmem;
-
-    if (warp >= 16) {
-        reg_dec<TC_REGS_OTHER>();   // the whole fifth warpgroup gives registers to the softmax warpgroups
-        if (warp == TC_TMA_WARP) {
-            // ------------------------------------------------------------ TMA producer (the rest of the tiles)
-            if (cnt > 0 && !ptx::mbar_wait(bar(BAR_Q), 0)) *abort_flag = 1;
-            for (int i = n_early; i < n_loads && !*abort_flag; ++i) {
-                const int slot = i % TC_SLOTS, use = i / TC_SLOTS;
-                if (use > 0 && !ptx::mbar_wait(bar(BAR_KV_EMPTY + slot), (use - 1) & 1)) { *abort_flag = 1; break; }
-                if (lane == 0) issue_kv(i);
-                __syncwarp();
+        if (lane == 0 && cnt > TC_EARLY) {
+            // the other tiles are requested once the query tile has landed, so that what the first MMAs need is
+            // not queued behind tiles that are needed later
+            if (!ptx::mbar_wait(bar(BAR_QFULL), 0)) give_up();
+            int issued = TC_EARLY;
+            for (int j = TC_EARLY; j < cnt && !*abort_flag; ++j) {
+                if (j >= TC_STAGES) {   // the slot's previous tile has been consumed by the tensor core
+                    const uint32_t par = ((j / TC_STAGES) - 1) & 1;
+                    if (!ptx::mbar_wait(bar(BAR_KFREE + j % TC_STAGES), par)) { give_up(); break; }
+                    issue_k(j);
+                    if (!ptx::mbar_wait(bar(BAR_VFREE + j % TC_STAGES), par)) { give_up(); break; }
+                    issue_v(j);
+                } else {
+                    issue_k(j);
+                    issue_v(j);
+                }
+                issued = j + 1;
             }
-        } else if (warp == TC_MMA_WARP) {
-            // ------------------------------------------------------------ MMA issuer
-            auto issue_S = [&](int t, int j) {
-                const uint32_t kbase = ring + ((2 * j) % TC_SLOTS) * TC_TILE_BYTES;
-                const uint32_t qbase = q_smem + t * TC_TILE_BYTES;
+            if (*abort_flag) {
+                // give every copy still in flight a bounded chance to land before the CTA can exit
+                ptx::mbar_wait(bar(BAR_QFULL), 0);
+                for (int j = max(0, issued - TC_STAGES); j < issued; ++j) {
+                    ptx::mbar_wait(bar(BAR_KFULL + j % TC_STAGES), (j / TC_STAGES) & 1);
+                    ptx::mbar_wait(bar(BAR_VFULL + j % TC_STAGES), (j / TC_STAGES) & 1);
+                }
+            }
+        }
+        __syncwarp();
+        ptx::cluster_arrive();
+    } else if (warp == TC_RELAY_WARP) {
+        // ------------------------------------------------------------ relay: this CTA's half has landed
+        bool ok = true;
+        for (int j = 0; j < cnt && ok && !*abort_flag; ++j) {
+            const int s = j % TC_STAGES;
+            const uint32_t par = (j / TC_STAGES) & 1;
+            ok = ptx::mbar_wait(bar(BAR_KFULL + s), par);
+            if (!ok) break;
+            if (j >= 2 && j < 7) TRACE(1 + j);   // K(j) landed
+            if (lane == 0) ptx::mbar_arrive_remote(lead(BAR_KREADY + s));
+            if (j == 0) {
+                ok = ptx::mbar_wait(bar(BAR_QFULL), 0);
+                if (!ok) break;
+                if (lane == 0) ptx::mbar_arrive_remote(lead(BAR_QREADY));
+            }
+            ok = ptx::mbar_wait(bar(BAR_VFULL + s), par);
+            if (!ok) break;
+            // Rows of the V tile past the last valid key hold whatever the cache holds there; their P is
+            // zero, but 0 * NaN would still poison O: clear them before the tensor core reads.
+            const int valid = n_keys - tile_of(j) * TC_BN;
+            if (valid < TC_BN) {
+                unsigned char *vt = gbase + TC_OFF_V + s * TC_V_BYTES;   // [128 keys][128 bytes]
+                for (int e = valid * 8 + lane; e < TC_BN * 8; e += 32)
+                    reinterpret_cast<uint4 *>(vt)[e] = make_uint4(0u, 0u, 0u, 0u);
+                ptx::fence_proxy_async();
+            }
+            __syncwarp();
+            if (lane == 0) {
+                if (valid < TC_BN) ptx::mbar_arrive_remote_release(lead(BAR_VREADY + s));   // hands over the cleared rows
+                else ptx::mbar_arrive_remote(lead(BAR_VREADY + s));
+            }
+        }
+        if (!ok && lane == 0) give_up();
+        __syncwarp();
+        ptx::cluster_arrive();
+    } else if (warp == TC_MMA_WARP) {
+        // ------------------------------------------------------------ issuer of S = Q K^T (even CTA, one thread)
+        // Two threads issue the MMAs, one per kind, so that the scores of the next groups never wait behind a P that
+        // is still being written: this one follows the K groups and the completed O += P V, the other one (below)
+        // the V groups and the finished P tiles.
+        if (rank == 0 && lane == 0 && cnt > 0) {
+            // Operand descriptors are built once; an instruction then costs its issuing thread one 64-bit add
+            // per operand (the start-address field counts 16-byte units and never carries: shared-memory
+            // addresses stay below 256 KB).
+            const uint64_t dq0 = desc_kmajor(q_smem), dk0 = desc_kmajor(k_ring);
+            bool ok = ptx::mbar_wait(bar(BAR_QREADY), 0);
+            for (int j = 0; ok && j < cnt && !*abort_flag; ++j) {
+                // the K group of both CTAs has landed; the S buffer (with P over it) has been consumed by both
+                // streams' O += P V of group j - 2
+                ok = ptx::mbar_wait(bar(BAR_KREADY + j % TC_STAGES), (j / TC_STAGES) & 1) &&
+                     (j < 2 || ptx::mbar_wait(bar(BAR_ODONE + (j & 1)), ((j >> 1) - 1) & 1));
+                if (!ok) break;
+                if (j == 0) TRACE(2);   // Q and K_0 of both CTAs landed
+                if (j >= 1 && j < 9) TRACE(55 + j);   // S(j) issued
+                ptx::tc_fence_after();
+                const uint64_t dk = dk0 + (uint64_t)(((j % TC_STAGES) * TC_K_BYTES) >> 4);
+                const uint32_t d = tmem + TM_S + (uint32_t)(j & 1) * 128;
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t off = (kk / 4) * TC_HALF_BYTES + (kk % 4) * 32;
-                    ptx::mma_ss(tmem + t * 128, desc_kmajor(qbase + off), desc_kmajor(kbase + off), IDESC_QK, kk > 0);
+                    const uint64_t offq = (uint64_t)(((kk / 4) * TC_Q_HALF + (kk % 4) * 32) >> 4);
+                    const uint64_t offk = (uint64_t)(((kk / 4) * TC_K_HALF + (kk % 4) * 32) >> 4);
+                    ptx::mma_pair_ss(d, dq0 + offq, dk + offk, IDESC_QK, kk > 0);
                 }
-            };
-            auto issue_PV = [&](int t, int j) {
-                const uint32_t vbase = ring + ((2 * j + 1) % TC_SLOTS) * TC_TILE_BYTES;
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    ptx::mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, desc_nmajor(vbase + kk * 2048), IDESC_PV,
-                                j > 0 || kk > 0);
-            };
-            auto wait_kv = [&](int i) { return ptx::mbar_wait(bar(BAR_KV_FULL + i % TC_SLOTS), (i / TC_SLOTS) & 1); };
-            bool ok = cnt == 0 || (wait_kv(0) && ptx::mbar_wait(bar(BAR_Q), 0));
-            if (ok && cnt > 0) {
-                TRACE(2);   // Q and K_0 landed
-                ptx::tc_fence_after();
-                if (lane == 0) {
-                    issue_S(0, 0);
-                    ptx::tc_commit(bar(BAR_S + 0));
-                }
-                __syncwarp();
-                if (nt == 2) ok = ptx::mbar_wait(bar(BAR_Q + 1), 0);
-                ptx::tc_fence_after();
-                if (ok && lane == 0) {
-                    if (nt == 2) { issue_S(1, 0); ptx::tc_commit(bar(BAR_S + 1)); }
-                    ptx::tc_commit(bar(BAR_KV_EMPTY + 0));
-                }
-                __syncwarp();
+                ptx::tc_commit_pair(bar(BAR_SREADY + (j & 1)));
+                ptx::tc_commit_pair(peer(BAR_SREADY + (j & 1)));
             }
-            for (int j = 0; ok && j < cnt && !*abort_flag; ++j) {
-                const bool more = j + 1 < cnt;
-                ok = wait_kv(2 * j + 1);
-                if (!ok) break;
-                {
-                    // Rows of the V tile past the last valid key hold whatever the cache holds there; their
-                    // P is zero, but 0 * NaN would still poison O: clear them before the tensor core reads.
-                    const int valid = n_keys - (t_begin + j) * TC_BN;
-                    if (valid < TC_BN) {
-                        unsigned char *vt = tiles_gen + TC_Q_BYTES + ((2 * j + 1) % TC_SLOTS) * TC_TILE_BYTES;
-                        for (int e = lane; e < (TC_BN - valid) * 16; e += 32) {
-                            const int row = valid + e / 16, c16 = e % 16;     // 16 x 16 bytes per row: 8 per half
-                            *reinterpret_cast<uint4 *>(vt + (c16 / 8) * TC_HALF_BYTES + row * 128 + (c16 % 8) * 16) =
-                                make_uint4(0u, 0u, 0u, 0u);
-                        }
-                        ptx::fence_proxy_async();
-                        __syncwarp();
-                    }
-                }
-                ok = ptx::mbar_wait(bar(BAR_P + 0), j & 1);
-                if (!ok) break;
-                ptx::tc_fence_after();
-                if (lane == 0) { issue_PV(0, j); ptx::tc_commit(bar(BAR_O + 0)); }
-                __syncwarp();
-                if (more) {
-                    ok = wait_kv(2 * j + 2);
-                    if (!ok) break;
-                    ptx::tc_fence_after();
-                    if (lane == 0) { issue_S(0, j + 1); ptx::tc_commit(bar(BAR_S + 0)); }
-                    __syncwarp();
-                }
-                if (nt == 2) {
-                    ok = ptx::mbar_wait(bar(BAR_P + 1), j & 1);
-                    if (!ok) break;
-                    ptx::tc_fence_after();
-                    if (lane == 0) { issue_PV(1, j); ptx::tc_commit(bar(BAR_O + 1)); }
-                    __syncwarp();
-                }
-                if (lane == 0) {
-                    ptx::tc_commit(bar(BAR_KV_EMPTY + (2 * j + 1) % TC_SLOTS));   // V_j is free once its MMAs are done
-                    if (more) {
-                        if (nt == 2) { issue_S(1, j + 1); ptx::tc_commit(bar(BAR_S + 1)); }
-                        ptx::tc_commit(bar(BAR_KV_EMPTY + (2 * j + 2) % TC_SLOTS));
-                    }
-                }
-                __syncwarp();
-            }
-            if (ok && cnt > 0 && !*abort_flag) {
-                if (lane == 0) ptx::tc_commit(bar(BAR_FINAL));   // follows every tensor-core operation issued
-                __syncwarp();
-                ctx.final_committed = true;
-            }
-            if (!ok) *abort_flag = 1;
+            if (!ok) give_up();
         }
-        tc_epilogue<false>(p, ctx);
-    } else {
-        reg_inc<TC_REGS_SOFTMAX>();
-        if (warp / 8 < nt) {
-            // ------------------------------------------------------------ softmax warps of row tile t
-            // Thread (row, hf) owns keys [64 hf, 64 hf + 64) of its query row in every key tile.
-            const int t = warp / 8, hf = (warp / 4) & 1;
-            const int row = (warp % 4) * 32 + lane;
-            const int r = rows0 + t * 128 + row;
-            uint64_t alo = 0, ahi = 0;
-            if (r < p.M_rows) { alo = p.anc[(r / p.G) * 2]; ahi = p.anc[(r / p.G) * 2 + 1]; }
-            const uint32_t lane_base = (uint32_t)((warp % 4) * 32) << 16;
-            const uint32_t t_s = tmem + lane_base + t * 128 + hf * 64;          // this thread's 64 columns of S_t
-            const uint32_t t_p = tmem + lane_base + t * 128 + hf * 32;          // its 32 columns of P_t
-            const uint32_t t_o = tmem + lane_base + 256 + t * 128 + hf * 64;    // its 64 columns of O_t
-            __nv_bfloat16 *xmax = reinterpret_cast<__nv_bfloat16 *>(bar_region + TC_BAR_BYTES);   // [t][hf][row]
-            auto pair_sync = [&]() { asm volatile("bar.sync %0, 256;" ::"r"(2 + t) : "memory"); };  // the 256 threads of row tile t
-            float m_used = -INFINITY, l = 0.f;
+        __syncwarp();
+        ptx::cluster_arrive();
+    } else if (warp == TC_PV_WARP) {
+        // ------------------------------------------------------------ issuer of O += P V (even CTA, one thread)
+        if (rank == 0 && lane == 0 && cnt > 0) {
+            const uint64_t dv0 = desc_nmajor(v_ring);
             bool ok = true;
-            // visibility of the tree rows as 32-bit words: word q covers tree rows 32q .. 32q+31
-            auto anc_word = [&](int q) -> uint32_t {
-                if (q < 0) return 0xffffffffu;     // prefix rows are visible to every node
-                if (q == 0) return (uint32_t)alo;
-                if (q == 1) return (uint32_t)(alo >> 32);
-                if (q == 2) return (uint32_t)ahi;
-                if (q == 3) return (uint32_t)(ahi >> 32);
-                return 0u;                         // past the tree rows: nothing
-            };
-            // A thread whose wait ran out keeps going through the motions without waiting, so that
-            // the barriers it shares with the other half-row threads stay matched.
-            for (int j = 0; j < cnt; ++j) {
-                if (*abort_flag) ok = false;
-                if (ok) ok = ptx::mbar_wait(bar(BAR_S + t), j & 1);
-                if (warp % 8 == 0 && j < 6) TRACE(8 + t * 16 + j * 2);       // S_t(j) ready
+            for (int j = 0; ok && j < cnt && !*abort_flag; ++j) {
+                // the V group of both CTAs has landed and both streams' P are in tensor memory (the two streams finish
+                // a group at about the same time: their scores arrive together)
+                ok = ptx::mbar_wait(bar(BAR_VREADY + j % TC_STAGES), (j / TC_STAGES) & 1) &&
+                     ptx::mbar_wait(bar(BAR_PREADY + (j & 1)), (j >> 1) & 1);
+                if (!ok) break;
                 ptx::tc_fence_after();
-                // ---- this thread's half row of S in registers (raw scores; the scale is positive)
-                uint32_t sr[2][32];
-                ptx::tmem_ld32(t_s, sr[0]);
-                ptx::tmem_ld32(t_s + 32, sr[1]);
-                ptx::tmem_ld_wait();
-                const int key0 = (t_begin + j) * TC_BN + hf * 64;
-                if (key0 + 64 > L) {
-                    // the half tile overlaps the tree rows or the end of the cache: bit e of vis is column 32c + e
+                if (j < 8) TRACE(48 + j);   // O += P V of group j issued
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        const int a0 = key0 + c * 32 - L;        // tree row of the chunk's first column
-                        const int q = a0 >> 5, sh = a0 & 31;     // floor division
-                        const uint32_t vis = __funnelshift_r(anc_word(q), anc_word(q + 1), sh);
+                for (int t = 0; t < 2; ++t) {   // stream t: keys [64 t, 64 t + 64) of the group
+                    const uint64_t dv = dv0 + (uint64_t)(((j % TC_STAGES) * TC_V_BYTES + t * TC_HALF * 128) >> 4);
+                    const uint32_t a = tmem + TM_S + (uint32_t)(j & 1) * 128 + (uint32_t)t * 64;
+                    const uint32_t d = tmem + TM_O + (uint32_t)t * 128;
 #pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (!((vis >> e) & 1u)) sr[c][e] = 0xff800000u;   // -inf
-                    }
+                    for (int kk = 0; kk < TC_HALF / 16; ++kk)
+                        ptx::mma_pair_ts(d, a + kk * 8, dv + (uint64_t)((kk * 2048) >> 4), IDESC_PV, j > 0 || kk > 0);
                 }
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-                for (int c = 0; c < 2; ++c)
-#pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        mx0 = fmaxf(mx0, __uint_as_float(sr[c][e]));
-                        mx1 = fmaxf(mx1, __uint_as_float(sr[c][e + 1]));
-                        mx2 = fmaxf(mx2, __uint_as_float(sr[c][e + 2]));
-                        mx3 = fmaxf(mx3, __uint_as_float(sr[c][e + 3]));
-                    }
-                // The two halves need the same reference, not the exact maximum (P may reach 2^8):
-                // they exchange their maxima rounded to bf16 and both take the larger rounded value.
-                const __nv_bfloat16 own = __float2bfloat16_rn(fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
-                xmax[(t * 2 + hf) * 128 + row] = own;
-                pair_sync();   // also: both halves hold their S before anyone overwrites it with P
-                const float mxs = fmaxf(__bfloat162float(own), __bfloat162float(xmax[(t * 2 + (hf ^ 1)) * 128 + row]));
-                const float m_new = (j == 0 || mxs > m_used + TC_RESCALE_THRESHOLD) ? mxs : m_used;
-                // O holds sums relative to m_used: rescale it when the reference moves (rare)
-                const bool need = j > 0 && m_new != m_used && m_used != -INFINITY;
-                if (__any_sync(0xffffffffu, need)) {
-                    if (ok) ok = ptx::mbar_wait(bar(BAR_O + t), (j - 1) & 1);
-                    ptx::tc_fence_after();
-                    const float alpha = need ? ex2(m_used - m_new) : 1.f;
-#pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t o[16];
-                        ptx::tmem_ld16(t_o + c * 16, o);
-                        ptx::tmem_ld_wait();
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                        ptx::tmem_st16(t_o + c * 16, o);
-                    }
-                    ptx::tmem_st_wait();
-                    l *= alpha;
-                }
-                m_used = m_new;
-                const float m_eff = m_used == -INFINITY ? 0.f : m_used;
-                // ---- P = exp2(scale * S - m), partial row sum, bf16 P over the first 64 columns of S_t
-                float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int e = 0; e < 16; e += 2) {
-                        const float p0 = ex2(fmaf(__uint_as_float(sr[c][2 * e]), p.scale_log2, -m_eff));
-                        const float p1 = ex2(fmaf(__uint_as_float(sr[c][2 * e + 1]), p.scale_log2, -m_eff));
-                        const float p2 = ex2(fmaf(__uint_as_float(sr[c][2 * e + 2]), p.scale_log2, -m_eff));
-                        const float p3 = ex2(fmaf(__uint_as_float(sr[c][2 * e + 3]), p.scale_log2, -m_eff));
-                        l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-                        pk[e] = pack2_bf16(p0, p1);
-                        pk[e + 1] = pack2_bf16(p2, p3);
-                    }
-                    ptx::tmem_st16(t_p + c * 16, pk);
-                }
-                l += (l0 + l1) + (l2 + l3);
-                ptx::tmem_st_wait();
-                ptx::tc_fence_before();
-                ptx::mbar_arrive(bar(BAR_P + t));
-                if (warp % 8 == 0 && j < 6) TRACE(9 + t * 16 + j * 2);       // P_t(j) written
+                ptx::tc_commit_pair(bar(BAR_ODONE + (j & 1)));
+                ptx::tc_commit_pair(peer(BAR_ODONE + (j & 1)));
             }
-            // ---- hand over the partial of this row
-            if (cnt > 0) {
-                // every tensor-core read of the tile buffers must be over before they are reused
-                if (*abort_flag) ok = false;
-                if (ok) ok = ptx::mbar_wait(bar(BAR_FINAL), 0);
-                if (warp % 8 == 0) TRACE(40 + t);                            // all tensor-core work done
-                ptx::tc_fence_after();
-            }
-            // the row sum is the sum of the two halves' sums
-            float *lx = reinterpret_cast<float *>(tiles_gen + TC_WBUF_OFF);   // [t][hf][row], free once the tiles are
-            lx[(t * 2 + hf) * 128 + row] = l;
-            pair_sync();
-            l += lx[(t * 2 + (hf ^ 1)) * 128 + row];
-            const bool have_o = cnt > 0 && ok;
-            {
-                // park this thread's 64 columns of O / l as bf16: chunk j at position j ^ (row & 15); an empty
-                // split parks zeros
-                unsigned char *dst = tiles_gen + (t * 128 + row) * TC_ROW_BYTES;
-                const int sw = (t * 128 + row) & 15;
-                const float inv_l = have_o && l > 0.f ? 1.f / l : 0.f;
-#pragma unroll 1
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t o[32];
-                    if (have_o) {
-                        ptx::tmem_ld32(t_o + c * 32, o);
-                        ptx::tmem_ld_wait();
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) o[e] = 0u;
-                    }
-#pragma unroll
-                    for (int e = 0; e < 32; e += 8) {
-                        uint4 pk;
-                        pk.x = pack2_bf16(__uint_as_float(o[e]) * inv_l, __uint_as_float(o[e + 1]) * inv_l);
-                        pk.y = pack2_bf16(__uint_as_float(o[e + 2]) * inv_l, __uint_as_float(o[e + 3]) * inv_l);
-                        pk.z = pack2_bf16(__uint_as_float(o[e + 4]) * inv_l, __uint_as_float(o[e + 5]) * inv_l);
-                        pk.w = pack2_bf16(__uint_as_float(o[e + 6]) * inv_l, __uint_as_float(o[e + 7]) * inv_l);
-                        *reinterpret_cast<uint4 *>(dst + (((hf * 8 + c * 4 + e / 8) ^ sw) << 4)) = pk;
-                    }
-                }
-                if (hf == 0) park_ml[t * 128 + row] = make_float2(m_used, l);   // (-inf, 0) for an empty split
-                ptx::fence_proxy_async();   // the bulk copy out of shared memory must see these stores
-            }
-            if (!ok) *abort_flag = 1;
+            if (!ok || *abort_flag) give_up();
+            // Every S group is read before its P is written and every P is consumed by one of the MMAs above, so when
+            // these have completed all tensor-core work of the pair has (on the error path the other issuer's MMAs may
+            // still run: the final cluster barrier is only passed by threads that have stopped signalling).
+            ptx::tc_commit_pair(bar(BAR_FINAL));
+            ptx::tc_commit_pair(peer(BAR_FINAL));
+            if (!ok || *abort_flag) ptx::mbar_wait(bar(BAR_FINAL), 0);   // let what was issued finish
         }
-        tc_epilogue<true>(p, ctx);
+        __syncwarp();
+        ptx::cluster_arrive();
+    } else {
+        // ------------------------------------------------------------ softmax warps
+        // Thread (row, st) owns query row `row` in stream st: keys [64 st, 64 st + 64) of every group.
+        const int qd = warp & 3, st = warp >> 2;
+        const int row = qd * 32 + lane;
+        const int r = rows0 + row;
+        uint64_t alo = 0, ahi = 0;
+        if (r < p.M_rows) { alo = p.anc[(r / p.G) * 2]; ahi = p.anc[(r / p.G) * 2 + 1]; }
+        const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
+        const uint32_t t_s = tmem + lane_base + TM_S + st * 64;   // + 128 for the odd groups; P goes over its first 32 columns
+        const uint32_t t_o = tmem + lane_base + TM_O + st * 128;
+        auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(2 + qd) : "memory"); };   // the two warps that share these rows
+        float m_used = -INFINITY, l = 0.f;
+        bool ok = true;
+        // visibility of the tree rows as 32-bit words: word w covers tree rows 32 w .. 32 w + 31
+        auto anc_word = [&](int w) -> uint32_t {
+            if (w < 0) return 0xffffffffu;     // prefix rows are visible to every node
+            if (w == 0) return (uint32_t)alo;
+            if (w == 1) return (uint32_t)(alo >> 32);
+            if (w == 2) return (uint32_t)ahi;
+            if (w == 3) return (uint32_t)(ahi >> 32);
+            return 0u;                         // past the tree rows: nothing
+        };
+        const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+        for (int j = 0; j < cnt; ++j) {
+            if (!ok || !ptx::mbar_wait(bar(BAR_SREADY + (j & 1)), (j >> 1) & 1)) { if (ok && lane == 0) give_up(); ok = false; }
+            if (qd == 0 && j < 8) TRACE(8 + j * 4 + st * 2);       // S(j) ready
+            ptx::tc_fence_after();
+            uint32_t sr[64];
+            ptx::tmem_ld32(t_s + (j & 1) * 128, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+            ptx::tmem_ld32(t_s + (j & 1) * 128 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
+            // S of group j is complete: its K slot is free; so are (the S buffer was only refilled after them) both
+            // streams' O += P V of group j - 2: that group's V slot is free
+            if (lane == 0) {
+                ptx::mbar_arrive(bar(BAR_KFREE + j % TC_STAGES));
+                if (j >= 2) ptx::mbar_arrive(bar(BAR_VFREE + (j - 2) % TC_STAGES));
+            }
+            ptx::tmem_ld_wait_for(*reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+            ptx::tmem_ld_wait_for(*reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
+            const int key0 = tile_of(j) * TC_BN + st * TC_HALF;
+            if (key0 + TC_HALF > L) {
+                // the tile overlaps the tree rows or the end of the cache: bit e of vis[h] is column 32 h + e
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int a0 = key0 + h * 32 - L;        // tree row of the half's first column
+                    const int w = a0 >> 5, sh = a0 & 31;     // floor division
+                    const uint32_t vis = __funnelshift_r(anc_word(w), anc_word(w + 1), sh);
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (!((vis >> e) & 1u)) sr[h * 32 + e] = 0xff800000u;   // -inf
+                }
+            }
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int e = 0; e < 64; e += 8)
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    mx[k] = ptx::fmax3(mx[k], __uint_as_float(sr[e + 2 * k]), __uint_as_float(sr[e + 2 * k + 1]));
+            const float mxs = fmaxf(ptx::fmax3(mx[0], mx[1], mx[2]), mx[3]) * p.scale_log2;   // the scale is positive
+            const float m_new = (j == 0 || mxs > m_used + TC_RESCALE_THRESHOLD) ? mxs : m_used;
+            // O of this stream holds sums relative to m_used: rescale it when the reference moves (rare), once the
+            // stream's O += P V of group j - 1 has completed
+            const bool need = j > 0 && m_new != m_used && m_used != -INFINITY;
+            if (__any_sync(0xffffffffu, need)) {
+                if (ok && !ptx::mbar_wait(bar(BAR_ODONE + ((j - 1) & 1)), ((j - 1) >> 1) & 1)) { ok = false; if (lane == 0) give_up(); }
+                ptx::tc_fence_after();
+                const float alpha = need ? ex2(m_used - m_new) : 1.f;
+#pragma unroll 1
+                for (int h = 0; h < 4; ++h) {
+                    uint32_t o[32];
+                    ptx::tmem_ld32(t_o + h * 32, o);
+                    ptx::tmem_ld_wait_for(o);
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                    ptx::tmem_st32(t_o + h * 32, o);
+                }
+                ptx::tmem_st_wait();
+                l *= alpha;
+            }
+            m_used = m_new;
+            const float m_eff = m_used == -INFINITY ? 0.f : m_used;
+            // ---- P = exp2(scale * S - m) with its row sum (two values per instruction where the instruction set
+            //      has packed forms), bf16 P into tensor memory over this thread's own scores
+            const float2 nm2 = make_float2(-m_eff, -m_eff);
+            float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
+            uint32_t pk[32];
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+                const float2 x01 = __ffma2_rn(make_float2(__uint_as_float(sr[2 * e]), __uint_as_float(sr[2 * e + 1])), sc2, nm2);
+                const float2 x23 = __ffma2_rn(make_float2(__uint_as_float(sr[2 * e + 2]), __uint_as_float(sr[2 * e + 3])), sc2, nm2);
+                const float2 p01 = make_float2(ex2(x01.x), ex2(x01.y)), p23 = make_float2(ex2(x23.x), ex2(x23.y));
+                la = __fadd2_rn(la, p01);
+                lb = __fadd2_rn(lb, p23);
+                pk[e] = pack2_bf16(p01.x, p01.y);
+                pk[e + 1] = pack2_bf16(p23.x, p23.y);
+            }
+            l += (la.x + la.y) + (lb.x + lb.y);
+            ptx::tmem_st32(t_s + (j & 1) * 128, pk);
+            ptx::tmem_st_wait();
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_remote(lead(BAR_PREADY + (j & 1)));
+            if (qd == 0 && j < 8) TRACE(9 + j * 4 + st * 2);       // P(j) written by this warp
+        }
+        // ---- all tensor-core work of the pair is done
+        if (cnt > 0) {
+            if (*abort_flag) ok = false;
+            if (ok && !ptx::mbar_wait(bar(BAR_FINAL), 0)) { ok = false; if (lane == 0) give_up(); }
+            if (warp == 0) TRACE(40);
+            ptx::tc_fence_after();
+        }
+        __syncwarp();
+        ptx::cluster_arrive_relaxed();   // nothing more goes to the peer from this thread
+        if (warp == 0) TRACE(3);
+        // ---- the two streams of a row are merged: O = (w0 O0 + w1 O1) / (w0 l0 + w1 l1) with w_t = exp2(m_t - m);
+        //      a stream that had no tile has (m, l) = (-inf, 0) and its accumulator is not read
+        ml_x[st * 128 + row] = make_float2(m_used, l);
+        pair_sync();
+        if (warp == 0) TRACE(4);
+        const float2 other = ml_x[(st ^ 1) * 128 + row];
+        const float m_all = fmaxf(m_used, other.x);
+        const float w_own = m_used == -INFINITY ? 0.f : ex2(m_used - m_all);
+        const float w_oth = other.x == -INFINITY ? 0.f : ex2(other.x - m_all);
+        const float l_all = w_own * l + w_oth * other.y;
+        const float inv_l = ok && l_all > 0.f ? 1.f / l_all : 0.f;
+        const float w0 = (st == 0 ? w_own : w_oth) * inv_l, w1 = (st == 0 ? w_oth : w_own) * inv_l;
+        const bool have0 = ok && cnt > 0;   // both streams had a tile in every group
+        // ---- this thread's 64 columns ([64 st, 64 st + 64)) as bf16 into the staging area (the Q tile is no longer
+        //      needed): 16-byte chunk j of row r sits at chunk position j ^ (r & 15), so that both the one-row-per-lane
+        //      stores here and the one-row-per-half-warp loads below are free of bank conflicts
+        unsigned char *stage = gbase;
+        {
+            uint32_t o0[2][32], o1[2][32];   // this thread's 64 columns of O of stream 0 and of stream 1
+            if (have0) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    ptx::tmem_ld32(tmem + lane_base + TM_O + (uint32_t)(st * 64 + h * 32), o0[h]);
+                    ptx::tmem_ld32(tmem + lane_base + TM_O + 128 + (uint32_t)(st * 64 + h * 32), o1[h]);
+                }
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    ptx::tmem_ld_wait_for(o0[h]);
+                    ptx::tmem_ld_wait_for(o1[h]);
+                }
+            }
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                float v[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    v[e] = have0 ? fmaf(__uint_as_float(o1[h][e]), w1, __uint_as_float(o0[h][e]) * w0) : 0.f;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    uint4 u;
+                    u.x = pack2_bf16(v[8 * e], v[8 * e + 1]);
+                    u.y = pack2_bf16(v[8 * e + 2], v[8 * e + 3]);
+                    u.z = pack2_bf16(v[8 * e + 4], v[8 * e + 5]);
+                    u.w = pack2_bf16(v[8 * e + 6], v[8 * e + 7]);
+                    *reinterpret_cast<uint4 *>(stage + row * 256 + (((st * 8 + h * 4 + e) ^ (row & 15)) << 4)) = u;
+                }
+            }
+        }
+        auto out_ptr = [&](int rr) {   // the 128 output values of query-block row rr
+            const int node = rr / p.G, hq = g * p.G + rr % p.G;
+            return p.out + (((size_t)b * p.T + node) * p.Hq + hq) * 128;
+        };
+        const int grp = blockIdx.z * gridDim.y + blockIdx.y;
+        const size_t slab0 = (size_t)grp * p.nsplit;     // first slab (256 rows) of this query block
+        const int slab_row0 = (int)rank * 128;
+        const int ch = lane & 15, hs = lane >> 4;
+        if (warp == 0) TRACE(5);
+        pair_sync();   // the rows of this quarter of the tile are staged
+        if (warp == 0) TRACE(6);
+        // what the merge below needs, computed while the stores are on their way
+        const int rows_per = (128 + p.nsplit - 1) / p.nsplit;
+        const int row_begin = split * rows_per;
+        const int n_my = max(0, min(128, row_begin + rows_per) - row_begin);
+        if (have_rows && !over) {
+            // ---- rows leave as whole 256-byte rows, two per warp instruction: warp (qd, st) takes rows 32 qd + 16 st ..
+            uint4 v[8];
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+                const int srow = qd * 32 + st * 16 + it * 2 + hs;
+                v[it] = *reinterpret_cast<const uint4 *>(stage + srow * 256 + ((ch ^ (srow & 15)) << 4));
+            }
+            if (p.nsplit == 1) {
+#pragma unroll
+                for (int it = 0; it < 8; ++it) {
+                    const int srow = qd * 32 + st * 16 + it * 2 + hs;
+                    if (rows0 + srow < p.M_rows) *reinterpret_cast<uint4 *>(out_ptr(rows0 + srow) + ch * 8) = v[it];
+                }
+            } else {
+                uint4 *dst = reinterpret_cast<uint4 *>(p.ws_o + ((slab0 + split) * 256 + slab_row0 + qd * 32 + st * 16 + hs) * 128 + ch * 8);
+#pragma unroll
+                for (int it = 0; it < 8; ++it) __stcg(dst + it * 2 * 16, v[it]);   // two rows of 16 chunks further each time
+            }
+        }
+        if (warp == 0) TRACE(7);
+        if (p.nsplit > 1 && have_rows && !over) {
+            // ---- publish this split's rows, then combine a slice of the rows of all splits
+            if (st == 0) __stcg(p.ws_ml + (slab0 + split) * 256 + slab_row0 + row, make_float2(m_all, l_all));
+            softmax_sync();   // every softmax thread's stores precede the release below
+            int32_t *arrive = p.arrive + grp * 2 + rank, *depart = p.depart + grp * 2 + rank;
+            if (threadIdx.x == 0) {
+                TRACE(44);   // partial written
+                __threadfence();
+                TRACE(41);   // fence done
+                asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(arrive) : "memory");
+                // relaxed polls (a round trip to L2 each), one acquire when the counter is full
+                const long long t0 = clock64();
+                while (*reinterpret_cast<volatile int32_t *>(arrive) < p.nsplit)
+                    if (clock64() - t0 > ptx::WAIT_CYCLE_LIMIT) { atomicExch(p.dev_error, MTV_ERR_TIMEOUT); break; }
+                (void)ld_acquire(arrive);
+                TRACE(45);   // everybody arrived
+            }
+            softmax_sync();
+            // This CTA has seen the counter full.  The last one to say so puts both counters back to zero at the end
+            // (nobody polls them any more; the next call cannot start before this kernel has ended); the atomic is
+            // issued here so that its round trip overlaps the merge.
+            int departed = 0;
+            if (threadIdx.x == 0) departed = atomicAdd(depart, 1);
+            // half a warp per row, lane = 16-byte chunk of the row; all loads of a row first, then the arithmetic: one
+            // round trip to L2 per pass, and with up to 16 rows per pass one pass for up to 8 splits
+            for (int rl0 = warp * 2; rl0 < n_my; rl0 += 2 * TC_SOFTMAX_WARPS) {   // warp-uniform trip count: shuffles inside
+                const bool mine = rl0 + hs < n_my;
+                const int rl = mine ? rl0 + hs : rl0;            // the odd half warp may have no row: it repeats its neighbour's loads
+                const int srow = slab_row0 + row_begin + rl;     // row inside a slab
+                const int rr = blk * 256 + srow;                 // row inside the (sequence, KV head) block
+                const __nv_bfloat16 *src = p.ws_o + (slab0 * 256 + srow) * 128 + ch * 8;
+                float acc[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+                float m = -INFINITY, wsum = 0.f;
+                for (int sp0 = 0; sp0 < p.nsplit; sp0 += 16) {   // (m, l) of up to 16 splits: lane ch holds split sp0 + ch
+                    float2 ml = make_float2(-INFINITY, 0.f);
+                    if (sp0 + ch < p.nsplit) ml = __ldcg(p.ws_ml + (slab0 + sp0 + ch) * 256 + srow);
+                    uint4 v[16];
+#pragma unroll
+                    for (int u = 0; u < 16; ++u)
+                        v[u] = sp0 + u < p.nsplit ? __ldcg(reinterpret_cast<const uint4 *>(src + (size_t)(sp0 + u) * 256 * 128))
+                                                  : make_uint4(0u, 0u, 0u, 0u);
+                    if (warp == 0 && sp0 == 0) TRACE(42);   // loads issued
+                    // running maximum over the chunks of 16 splits (a second chunk rescales what has been summed)
+                    float mc = ml.x;
+#pragma unroll
+                    for (int o = 8; o > 0; o >>= 1) mc = fmaxf(mc, __shfl_xor_sync(0xffffffffu, mc, o));
+                    const float m_new = fmaxf(m, mc);
+                    const float resc = m == -INFINITY ? 0.f : ex2(m - m_new);
+                    const float w = ml.x == -INFINITY ? 0.f : ex2(ml.x - m_new) * ml.y;   // unnormalised weight of split sp0 + ch
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[e] *= resc;
+                    m = m_new;
+#pragma unroll
+                    for (int u = 0; u < 16; ++u) {
+                        const float wu = __shfl_sync(0xffffffffu, w, (lane & 16) | u);
+                        const uint32_t vw[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            acc[2 * e] = fmaf(wu, __uint_as_float(vw[e] << 16), acc[2 * e]);
+                            acc[2 * e + 1] = fmaf(wu, __uint_as_float(vw[e] & 0xffff0000u), acc[2 * e + 1]);
+                        }
+                    }
+                    // the weights' sum rides along in every lane: sum over the half warp, folded into the same recurrence
+                    float ws = w;
+#pragma unroll
+                    for (int o = 8; o > 0; o >>= 1) ws += __shfl_xor_sync(0xffffffffu, ws, o);
+                    wsum = wsum * resc + ws;
+                }
+                if (warp == 0) TRACE(43);   // rows of all splits arrived and combined
+                const float inv = wsum > 0.f ? 1.f / wsum : 0.f;
+                if (mine && rr < p.M_rows)
+                    *reinterpret_cast<uint4 *>(out_ptr(rr) + ch * 8) =
+                        make_uint4(pack2_bf16(acc[0] * inv, acc[1] * inv), pack2_bf16(acc[2] * inv, acc[3] * inv),
+                                   pack2_bf16(acc[4] * inv, acc[5] * inv), pack2_bf16(acc[6] * inv, acc[7] * inv));
+            }
+            if (threadIdx.x == 0 && departed == p.nsplit - 1) {
+                *arrive = 0;
+                *depart = 0;
+                __threadfence();
+            }
+            if (warp == 0) TRACE(46);   // merge done
+        }
     }
+
+    // ---- nobody leaves while the pair's tensor-core work may still read its shared memory, write its
+    //      tensor memory or arrive on its barriers: every thread arrived on the cluster barrier a second
+    //      time when it had sent the peer its last signal, and waits here for the peer's threads
+    ptx::tc_fence_before();
+    cta_sync();
+    ptx::cluster_wait();
+    ptx::tc_fence_after();
+    if (warp == TC_MMA_WARP) ptx::tmem_dealloc_pair(tmem, 512);
+    if (warp == 0) TRACE(47);
 }
 
 // ---------------------------------------------------------------------------------------- host
@@ -699,36 +745,29 @@ static bool encode_map(CUtensorMap *map, const void *base, const cuuint64_t dims
 bool attn_tc_eligible(int D, int G) { return D == 128 && (G == 1 || G == 2 || G == 4 || G == 8); }
 
 static int tc_prepare() {
-    static bool done = false;
-    if (!done) {
+    constexpr int MAX_DEV = 64;
+    static bool done[MAX_DEV] = {false};
+    int dev = 0;
+    MTV_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEV || !done[dev]) {
         MTV_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
-        // the register rebalancing inside the kernel assumes the pool of a 168-register launch
-        cudaFuncAttributes fa;
-        MTV_CUDA_CHECK(cudaFuncGetAttributes(&fa, tree_attn_tc_kernel));
-        if (fa.numRegs < TC_REGS_LAUNCH) {
-            set_last_error("tree_attn_tc_kernel was built with too few registers for its setmaxnreg targets", cudaErrorInvalidValue);
-            return MTV_ERR_CUDA;
-        }
-        done = true;
+        if (dev >= 0 && dev < MAX_DEV) done[dev] = true;
     }
     return MTV_OK;
 }
 
-// Number of key splits of a problem: as many as keep the whole grid within one wave of SMs
-// (one CTA per SM), at most one per key tile, at most TC_MAX_SPLITS.  More than one split needs
-// a merge counter per query block.
-int attn_tc_plan(int T, int G, int B, int Hkv, int Lcap, int *n_rt_out) {
-    const int n_rt = (T * G + 255) / 256;
-    const long base = (long)B * Hkv * n_rt;
+// Number of key splits of a problem: as many as keep the whole grid within one wave of CTA pairs (one CTA
+// per SM), at most one per key tile, at most TC_MAX_SPLITS.  More than one split needs two merge counters
+// per query block.
+int attn_tc_plan(int T, int G, int B, int Hkv, int Lcap, int *n_blk_out) {
+    const int n_blk = (T * G + 255) / 256;
+    const long base = (long)B * Hkv * n_blk;
     const int tiles = (Lcap + TC_BN - 1) / TC_BN;
-    long ns = sm_count() / base;
+    long ns = (sm_count() / 2) / base;
     if (ns > tiles) ns = tiles;
     if (ns > TC_MAX_SPLITS) ns = TC_MAX_SPLITS;
-#ifdef TC_FORCE_NSPLIT
-    ns = TC_FORCE_NSPLIT;
-#endif
-    if (ns < 1 || base > TC_MAX_GROUPS) ns = 1;
-    if (n_rt_out) *n_rt_out = n_rt;
+    if (ns < 1 || base * 2 > TC_MAX_COUNTERS) ns = 1;
+    if (n_blk_out) *n_blk_out = n_blk;
     return (int)ns;
 }
 
@@ -747,29 +786,26 @@ int launch_tree_attn_tc(const mtv_tree *tree, int B, int Hq, int Hkv, const __nv
     {
         const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)Lcap, (cuuint64_t)Hkv, (cuuint64_t)B};
         const cuuint64_t str[3] = {(cuuint64_t)st * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
-        const cuuint32_t box[4] = {64, 128, 1, 1};
-        if (!encode_map(&k_map, k, dims, str, box) || !encode_map(&v_map, v, dims, str, box)) return MTV_ERR_CUDA;
+        const cuuint32_t kbox[4] = {64, TC_BN / 2, 1, 1}, vbox[4] = {64, TC_BN, 1, 1};
+        if (!encode_map(&k_map, k, dims, str, kbox) || !encode_map(&v_map, v, dims, str, vbox)) return MTV_ERR_CUDA;
     }
     if (tc_prepare() != MTV_OK) return MTV_ERR_CUDA;
     TcParams p;
     p.seq_lens = seq_lens; p.anc = tree->d_anc; p.out = out; p.status = status; p.dev_error = tree->d_error;
     p.ws_o = reinterpret_cast<__nv_bfloat16 *>(ws_o); p.ws_ml = reinterpret_cast<float2 *>(ws_ml);
-    p.arrive = tree->d_counters; p.depart = tree->d_counters + TC_MAX_GROUPS;
+    p.arrive = tree->d_counters; p.depart = tree->d_counters + TC_MAX_COUNTERS;
     p.scale_log2 = scale_log2;
     p.T = T; p.G = G; p.Hq = Hq; p.Hkv = Hkv; p.Lcap = Lcap;
-    p.nsplit = attn_tc_plan(T, G, B, Hkv, Lcap, &p.n_rt);
+    p.nsplit = attn_tc_plan(T, G, B, Hkv, Lcap, &p.n_blk);
     p.M_rows = T * G;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.nsplit, Hkv * p.n_rt, B);
+    cfg.gridDim = dim3(2 * p.nsplit, Hkv * p.n_blk, B);   // the kernel's cluster is (2, 1, 1): a CTA pair
     cfg.blockDim = dim3(TC_THREADS, 1, 1);
     cfg.dynamicSmemBytes = TC_SMEM_BYTES;
     cfg.stream = stream;
     // Launched as a programmatic dependent of the previous kernel in the stream (the kernel itself
     // waits for that kernel before it reads anything), which hides most of the launch latency when
-    // attention calls follow each other.  Not a cooperative launch: that costs about 2 us per
-    // launch; the grid never exceeds one CTA per SM, so its CTAs are resident together whenever the
-    // device is not shared with another long-running kernel, and the wait for the other splits is
-    // bounded in any case.
+    // attention calls follow each other.
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
