@@ -40,6 +40,9 @@ def parse():
     ap.add_argument("--no-taps", action="store_true", help="skip per-kernel event timing")
     ap.add_argument("--launch", default="graph", choices=["graph", "stream"],
                     help="timed steps: replay of one captured CUDA graph per step, or plain stream launches")
+    ap.add_argument("--repeats", type=int, default=5, help="timed repeats of --steps; the median is reported")
+    ap.add_argument("--no-other-workloads", action="store_true", help="skip the short runs of the other four configurations")
+    ap.add_argument("--no-parity-gate", action="store_true", help="skip the checks against the CPU checker before timing")
     ap.add_argument("--overhead-sweep", action="store_true",
                     help="instead of the step benchmark: time tree attention (T nodes) against single-token decode "
                          "attention (a root-only tree) over prefix lengths, the attention part of the paper's overhead ratio")
@@ -201,6 +204,72 @@ def build_problem(w, n_layers, device, seed=None):
 LAUNCHES_PER_STEP = lambda n_layers: 2 + n_layers + 2 + 2
 
 
+def workload_string(w, T, n_layers):
+    """The description of a workload, identical in both arms."""
+    return "%s: B=%d prefix=%s H=%d Hq/Hkv=%d/%d D=%d V=%d K=%d T=%d layers=%d" % (
+        w.name, w.B, w.L_lo if w.L_lo == w.L_hi else "U[%d,%d]" % (w.L_lo, w.L_hi), w.H, w.Hq, w.Hkv, w.D, w.V,
+        w.K, T, n_layers)
+
+
+class ParityError(RuntimeError):
+    pass
+
+
+def parity_gate(w, P, n_layers, rows=96):
+    """Checks of this run's own results against the CPU checker, before anything is timed: sampled attention rows
+    of one layer, the tree tokens of the heads pass, and the acceptance outputs of one whole step.  Raises ParityError."""
+    import torch
+    from oracle import reference as ref
+    from oracle import tree as otree
+    from paper_2603_03383_b200 import binding
+    tree, B, T = P["tree"], w.B, P["tree"].T
+    nodes = otree.cartesian(w.topk) if w.tree == "cartesian" else otree.rank_prior(w.K, w.T, w.R_max)
+    tb = otree.tables(nodes, w.K)
+    t0 = time.perf_counter()
+    report = {}
+    # attention: sampled (sequence, node, head) rows of the last layer, against the cache as it is now
+    l = n_layers - 1
+    total = B * T * w.Hq
+    sel = sorted({(i * 2654435761) % total for i in range(rows)})
+    rws = [(r // (T * w.Hq), (r // w.Hq) % T, r % w.Hq) for r in sel]
+    out = torch.zeros_like(P["q_layers"][l])
+    binding.tree_verify_attention(tree, P["q_layers"][l], P["k_list"][l], P["v_list"][l], P["seq_lens0"], out, P["ws"])
+    torch.cuda.synchronize()
+    want = ref.tree_attention(P["q_layers"][l].cpu(), P["k_list"][l].cpu(), P["v_list"][l].cpu(), P["lens"], tb["mask"],
+                              rows=rws)
+    got = torch.stack([out[b, i, h].cpu() for b, i, h in rws]).double()
+    err = (got - want).abs().max().item()
+    tol = 1e-2 * want.abs().max().item() + 1e-3
+    if not err <= tol:
+        raise ParityError("attention rows: max |err| %.3e above %.3e" % (err, tol))
+    report["attention"] = "%d rows of layer %d: max |err| %.2e <= %.2e" % (len(rws), l, err, tol)
+    # one whole step on the device
+    P["seq_lens"].copy_(P["seq_lens0"])
+    binding.mtv_verify_step(tree, P["args"])
+    torch.cuda.synchronize()
+    if any(P["status"].cpu().tolist()):
+        raise ParityError("status %s" % P["status"].cpu().tolist())
+    # tree tokens: the checker's heads + top-k + expansion on the same inputs
+    z = ref.heads_logits(P["hidden"].cpu(), P["W1"].cpu(), P["b1"].cpu(), P["W2"].cpu())
+    _, _, tt_ref, _ = ref.heads_candidates(z, P["root_tok"].cpu(), tb)
+    del z
+    if not torch.equal(P["tree_tok"].cpu(), tt_ref):
+        raise ParityError("tree_tok differs from the checker's")
+    report["tree_tok"] = "bit-exact (%d x %d)" % (B, T)
+    # acceptance: the checker on the stored logits, and the planted lengths
+    acc_ref = ref.tree_accept(ref.node_argmax(P["logits"].cpu()), tt_ref, tb)
+    for name in ("accept_len", "best_path", "acc_nodes", "acc_tok", "next_root"):
+        if not torch.equal(P[name].cpu(), acc_ref[name]):
+            raise ParityError("%s differs from the checker's" % name)
+    if not torch.equal(P["accept_len"].cpu(), P["planted"].to(torch.int32).cpu()):
+        raise ParityError("accept_len differs from the planted lengths")
+    if not torch.equal(P["seq_lens"].cpu(), P["lens"] + acc_ref["accept_len"] + 1):
+        raise ParityError("seq_lens not advanced by accept_len + 1")
+    report["acceptance"] = "bit-exact, equals the planted lengths %s" % P["planted"].tolist()
+    report["seconds"] = round(time.perf_counter() - t0, 2)
+    return report
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -217,6 +286,15 @@ def run_ours(args):
     P = build_problem(w, n_layers, dev, seed=rank_seed(w, rank))
     tree, a = P["tree"], P["args"]
     K_steps, W_steps = args.steps, max(args.warmup, 3)
+    gate = None
+    if rank == 0 and not args.no_parity_gate:
+        # nothing is timed, and no value printed, unless this run's own results match the CPU checker
+        try:
+            gate = parity_gate(w, P, n_layers)
+        except ParityError as e:
+            print(json.dumps({"metric": METRIC, "value": None, "unit": UNIT, "error": "parity gate failed: %s" % e,
+                              "config": {"workload": workload_string(w, tree.T, n_layers)}}))
+            sys.exit(1)
 
     def step():
         P["seq_lens"].copy_(P["seq_lens0"])          # shapes stay fixed from step to step
@@ -273,16 +351,20 @@ def run_ours(args):
         b1.record()
         barrier()
         attn_block_ms = b0.elapsed_time(b1) / (tap_steps * n_layers)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record()
-    for _ in range(K_steps):
-        run_step()
-    e1.record()
-    barrier()
-    ms_total = e0.elapsed_time(e1)
+    # the timed region: `repeats` runs of exactly K_steps steps, each bracketed by a barrier and a device synchronise;
+    # the reported time is the median run (max over ranks per run)
+    runs_ms = []
+    for _ in range(max(1, args.repeats)):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for _ in range(K_steps):
+            run_step()
+        e1.record()
+        barrier()
+        runs_ms.append(max_over_ranks(e0.elapsed_time(e1), world, dev))
     clocks = sampler.stop() if rank == 0 else None
-    ms_total = max_over_ranks(ms_total, world, dev)
+    ms_total = statistics.median(runs_ms)
     ms_step = ms_total / K_steps
     value = world * 1000.0 / ms_step
     mean_tokens = (P["accept_len"].float().mean().item() + 1.0)
@@ -321,9 +403,9 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W_steps,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": "%s: B=%d prefix=%s H=%d Hq/Hkv=%d/%d D=%d V=%d K=%d T=%d layers=%d" % (
-            w.name, w.B, w.L_lo if w.L_lo == w.L_hi else "U[%d,%d]" % (w.L_lo, w.L_hi), w.H, w.Hq, w.Hkv, w.D, w.V,
-            w.K, tree.T, n_layers),
+        "config": {"workload": workload_string(w, tree.T, n_layers),
+            "timing": "median of %d runs of %d steps (%s ms each)" % (
+                len(runs_ms), K_steps, ", ".join("%.1f" % r for r in runs_ms)),
             "l2": "inputs larger than L2: %.2f GB streamed per step, %d distinct KV caches" % (alg["step"] / 1e9, n_layers),
             "launch": ("one CUDA graph per step (captured mtv_verify_step), replayed" if args.launch == "graph"
                        else "stream launches through mtv_verify_step"), "seed": w.seed,
@@ -333,6 +415,7 @@ def run_ours(args):
                 "steps": e2e_steps},
         "gpu_launches": K_steps * LAUNCHES_PER_STEP(n_layers),
         "device_error": binding.mtv_device_error(tree, clear=False),
+        "parity_gate": gate if gate is not None else "skipped",
         "step_roofline": {"algorithmic_bytes": alg["step"], "achieved_gbs": alg["step"] / ms_step / 1e6,
                           "frac_of_measured": alg["step"] / ms_step / 1e6 / pk["hbm_gbs"],
                           "frac_of_8tbs": alg["step"] / ms_step / 1e6 / 8000.0},
@@ -378,12 +461,87 @@ def run_ours(args):
             "algorithmic_bytes": alg["step"] - alg["accept"] + lm_bytes,
             "frac_of_measured_hbm": (alg["step"] - alg["accept"] + lm_bytes) / lm_step_ms / 1e6 / pk["hbm_gbs"]}}
     if not args.no_cpu_baseline and world == 1:
-        out["cpu_baseline"] = cpu_baseline(w, P, n_layers, budget_s=25.0)
+        out["cpu_baseline"] = cpu_baseline(w, P, n_layers, budget_s=20.0)
+    if not args.no_other_workloads and world == 1:
+        del P
+        torch.cuda.empty_cache()
+        out["other_workloads"] = {}
+        for name in ("tiny", "short", "batched", "stress"):
+            if name != w.name:
+                out["other_workloads"][name] = quick_workload(name, n_layers, dev, pk)
     elif not args.no_cpu_baseline:
         out["cpu_baseline"] = None
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def quick_workload(name, n_layers, dev, pk, steps=5, repeats=3):
+    """A short measurement of one of the other configurations: whole steps (graph replay and plain stream launches:
+    their difference is the launch overhead), the attention call alone, and the roofline fractions that go with them.
+    Checked before timing: statuses, and the accepted lengths against the planted ones."""
+    import torch
+    from paper_2603_03383_b200 import binding, synth
+    w = synth.WORKLOADS[name]
+    P = build_problem(w, n_layers, dev)
+    tree, a = P["tree"], P["args"]
+
+    def step():
+        P["seq_lens"].copy_(P["seq_lens0"])
+        binding.mtv_verify_step(tree, a)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    checks = (not any(P["status"].cpu().tolist())) and torch.equal(P["accept_len"].cpu(), P["planted"].to(torch.int32).cpu())
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    torch.cuda.current_stream().wait_stream(side)
+
+    def timed(fn, n):
+        best = []
+        for _ in range(repeats):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(n):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            best.append(e0.elapsed_time(e1) / n)
+        return statistics.median(best)
+
+    graph.replay()
+    ms_graph = timed(graph.replay, steps)
+    ms_stream = timed(step, steps)
+
+    def attn_block():
+        for l in range(n_layers):
+            binding.tree_verify_attention(tree, P["q_layers"][l], P["k_list"][l], P["v_list"][l], P["seq_lens0"],
+                                          P["out_layers"][l], P["ws"])
+    attn_block()
+    attn_us = timed(attn_block, 3) * 1e3 / n_layers
+    alg = algorithmic_bytes(w, tree, n_layers, P["lens"].tolist())
+    T = tree.T
+    attn_flops = sum(4.0 * (L + T) * T * w.Hq * w.D for L in P["lens"].tolist())
+    res = {
+        "workload": workload_string(w, T, n_layers), "checks_passed": bool(checks),
+        "steps_per_s": 1000.0 / ms_graph, "ms_per_step": ms_graph, "ms_per_step_stream_launches": ms_stream,
+        "launch_overhead_share": max(0.0, (ms_stream - ms_graph) / ms_stream),
+        "step_frac_of_measured_hbm": alg["step"] / ms_graph / 1e6 / pk["hbm_gbs"],
+        "attn_us_per_call": attn_us,
+        "attn_frac_of_measured_hbm": alg["attn_per_layer"] / attn_us / 1e3 / pk["hbm_gbs"],
+        "attn_tflops": attn_flops / attn_us / 1e6,
+        "attn_frac_of_measured_bf16": attn_flops / attn_us / 1e6 / pk["bf16_tflops"],
+        "device_error": binding.mtv_device_error(tree, clear=False),
+    }
+    del P
+    torch.cuda.empty_cache()
+    return res
 
 
 def time_lm_head(tree, w, P, dev, iters=20):
@@ -562,9 +720,9 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": K_steps, "warmup": W_steps, "ms_per_step": full * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "%s: same shapes as the CUDA arm, layers=%d" % (w.name, n_layers),
-                   "note": "each step is a bounded sample scaled to a whole step; timed wall %.1f s" % wall},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "config": {"workload": workload_string(w, S["T"], n_layers)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": desc + "; timed wall %.1f s" % wall},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
