@@ -197,11 +197,11 @@ static __device__ __align__(256) unsigned char g_accept_scratch[ACCEPT_STATIC_SC
 // only a handle for the runtime, not an address a kernel could use, so the address is asked for
 // once per device (with that device current) and remembered.
 static int accept_scratch_address(unsigned long long **out) {
-    constexpr int MAX_DEVICES = 64;
-    static unsigned long long *cached[MAX_DEVICES] = {nullptr};
+    // (two host threads that meet on first use of a device both look the address up and store the same value)
+    static unsigned long long *cached[MTV_MAX_DEVICES] = {nullptr};
     int dev = 0;
     MTV_CUDA_CHECK(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= MAX_DEVICES) return MTV_ERR_UNSUPPORTED_SHAPE;
+    if (dev < 0 || dev >= MTV_MAX_DEVICES) return MTV_ERR_UNSUPPORTED_SHAPE;
     if (!cached[dev]) {
         void *ptr = nullptr;
         MTV_CUDA_CHECK(cudaGetSymbolAddress(&ptr, g_accept_scratch));

@@ -347,11 +347,12 @@ extern "C" int tree_verify_attention(const mtv_tree_t *tree, int B, int Hq, int 
         if (Lw.use_tc) return MTV_ERR_INVALID_ARG;   // a negative scale
         const dim3 grid(Lw.nsplit, Hkv * (Lw.m_rows / BM), B);
         const size_t smem = (size_t)4 * BN * D * 2;
-        static bool attr_done = false;
-        if (!attr_done) {
+        static PerDeviceOnce attr_once;
+        bool *attr_done = attr_once.flag();
+        if (!attr_done || !*attr_done) {
             MTV_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_partial_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * BN * 64 * 2));
             MTV_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_partial_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * BN * 128 * 2));
-            attr_done = true;
+            if (attr_done) *attr_done = true;
         }
         TapScope tap(MTV_KERNEL_ATTN_PARTIAL, st);
         if (D == 64) tree_attn_partial_kernel<64><<<grid, ATT_THREADS, smem, st>>>(p);

@@ -42,6 +42,8 @@
 // Build option -DMTV_TRACE: per-CTA cycle stamps of the phases through mtv_trace_set (development aid).
 #include <cuda.h>
 
+#include <cstring>
+#include <mutex>
 #include <type_traits>
 
 #include "common.cuh"
@@ -754,27 +756,65 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// 4-D bf16 tensor map with a 128-byte-swizzled box whose innermost extent is 64 elements.
+// 4-D bf16 tensor map with a 128-byte-swizzled box whose innermost extent is 64 elements.  Encoding a map costs the host
+// a microsecond or two and an attention call needs three, so encoded maps are kept in a small direct-mapped table keyed by
+// everything that goes into them (a decode loop passes the same caches and strides step after step).
+namespace {
+struct MapKey {
+    const void *base;
+    cuuint64_t dims[4], strides[3];
+    cuuint32_t box[4];
+    int device;
+};
+struct MapSlot {
+    MapKey key;
+    CUtensorMap map;
+    bool valid = false;
+};
+constexpr int MAP_SLOTS = 512;
+MapSlot g_map_slots[MAP_SLOTS];
+std::mutex g_map_mutex;
+}  // namespace
+
 static bool encode_map(CUtensorMap *map, const void *base, const cuuint64_t dims[4], const cuuint64_t strides_bytes[3],
                        const cuuint32_t box[4]) {
+    MapKey key;
+    memset(&key, 0, sizeof key);
+    key.base = base;
+    for (int i = 0; i < 4; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
+    for (int i = 0; i < 3; ++i) key.strides[i] = strides_bytes[i];
+    if (cudaGetDevice(&key.device) != cudaSuccess) key.device = -1;
+    const uint64_t h = ((uint64_t)(uintptr_t)base >> 8) * 0x9E3779B97F4A7C15ull + dims[1] * 0xC2B2AE3D27D4EB4Full + box[1] * 0x165667B19E3779F9ull;
+    MapSlot &slot = g_map_slots[(h >> 40) % MAP_SLOTS];
+    {
+        std::lock_guard<std::mutex> lock(g_map_mutex);
+        if (slot.valid && memcmp(&slot.key, &key, sizeof key) == 0) {
+            *map = slot.map;
+            return true;
+        }
+    }
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint32_t ones[4] = {1, 1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides_bytes, box, ones,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    if (fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides_bytes, box, ones,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    std::lock_guard<std::mutex> lock(g_map_mutex);
+    slot.key = key;
+    slot.map = *map;
+    slot.valid = true;
+    return true;
 }
 
 bool attn_tc_eligible(int D, int G) { return D == 128 && (G == 1 || G == 2 || G == 4 || G == 8); }
 
 static int tc_prepare() {
-    constexpr int MAX_DEV = 64;
-    static bool done[MAX_DEV] = {false};
-    int dev = 0;
-    MTV_CUDA_CHECK(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= MAX_DEV || !done[dev]) {
+    static PerDeviceOnce once;
+    bool *done = once.flag();
+    if (!done || !*done) {
         MTV_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
-        if (dev >= 0 && dev < MAX_DEV) done[dev] = true;
+        if (done) *done = true;
     }
     return MTV_OK;
 }

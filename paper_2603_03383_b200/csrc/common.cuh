@@ -72,7 +72,20 @@ struct AcceptWs {
 };
 AcceptWs accept_ws_layout(const mtv_tree *t, int B, int V);
 
-int sm_count();
+int sm_count();   // of the current device
+
+// Set-up that has to happen once per device (kernel attributes, symbol addresses): one flag per device ordinal.
+// Two host threads that meet on first use both do the set-up; it is idempotent.
+constexpr int MTV_MAX_DEVICES = 64;
+struct PerDeviceOnce {
+    bool done[MTV_MAX_DEVICES] = {};
+    // the current device's flag, or null if the device cannot be told (the caller then does the set-up every time)
+    bool *flag() {
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MTV_MAX_DEVICES) return nullptr;
+        return &done[dev];
+    }
+};
 
 // Optional per-kernel event taps (see mtv_set_kernel_taps).
 struct Tap {

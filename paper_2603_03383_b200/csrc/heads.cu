@@ -450,11 +450,12 @@ static int launch_heads(const mtv_tree *t, int B, int H, int V, const __nv_bfloa
     const VocabSmem S = vocab_smem_plan(NB, H, L.ctas_per_head);
     if (sm1 > VT_SMEM_MAX || S.total == 0) return MTV_ERR_UNSUPPORTED_SHAPE;
     if (NB > 1 && S.rows_per_stage < (NB >= 4 ? 4 : 2)) return MTV_ERR_UNSUPPORTED_SHAPE;   // rows too long for a block of rows per stage
-    static bool attr_done = false;
-    if (!attr_done) {
+    static PerDeviceOnce attr_once;
+    bool *attr_done = attr_once.flag();
+    if (!attr_done || !*attr_done) {
         MTV_CUDA_CHECK(cudaFuncSetAttribute(heads_resblock_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, VT_SMEM_MAX));
         MTV_CUDA_CHECK(cudaFuncSetAttribute(heads_vocab_topk_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, VT_SMEM_MAX));
-        attr_done = true;
+        if (attr_done) *attr_done = true;
     }
     int g1 = (t->K * H + HEADS_WARPS - 1) / HEADS_WARPS;
     const int cap = 4 * sm_count();

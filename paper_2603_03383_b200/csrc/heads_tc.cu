@@ -424,11 +424,12 @@ size_t heads_tc_xsplit_bytes(int K, int H) { return (size_t)K * HT_N * H * sizeo
 int launch_heads_tc(const mtv_tree *t, int B, int H, int V, const __nv_bfloat16 *hidden, const __nv_bfloat16 *W1,
                     const __nv_bfloat16 *b1, const __nv_bfloat16 *W2, const int32_t *root_tok, int32_t *cand,
                     float *cand_logit, int32_t *tree_tok, const HeadsWs &L, char *ws, cudaStream_t st) {
-    static bool attr_done = false;
-    if (!attr_done) {
+    static PerDeviceOnce attr_once;
+    bool *attr_done = attr_once.flag();
+    if (!attr_done || !*attr_done) {
         MTV_CUDA_CHECK(cudaFuncSetAttribute(heads_vocab_topk_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, HT_SMEM_BYTES));
         MTV_CUDA_CHECK(cudaFuncSetAttribute(heads_resblock_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, RT_SMEM_BYTES));
-        attr_done = true;
+        if (attr_done) *attr_done = true;
     }
     __nv_bfloat16 *xsplit = reinterpret_cast<__nv_bfloat16 *>(ws + L.xsplit_off);
     CUtensorMap w1_map, h_map, w2_map, x_map;

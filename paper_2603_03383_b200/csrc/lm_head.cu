@@ -281,12 +281,13 @@ extern "C" int lm_head_argmax(const mtv_tree_t *tree, int B, int H, int V, const
     p.n_stages = (int)((LM_SMEM_MAX - 1024) / p.stage_bytes);
     if (p.n_stages > LM_MAX_STAGES) p.n_stages = LM_MAX_STAGES;
     const size_t smem = 1024 + (size_t)p.n_stages * p.stage_bytes;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static PerDeviceOnce attr_once;
+    bool *attr_done = attr_once.flag();
+    if (!attr_done || !*attr_done) {
         MTV_CUDA_CHECK(cudaFuncSetAttribute(lm_head_argmax_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, LM_SMEM_MAX));
         MTV_CUDA_CHECK(cudaFuncSetAttribute(lm_head_argmax_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, LM_SMEM_MAX));
         MTV_CUDA_CHECK(cudaFuncSetAttribute(lm_head_argmax_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, LM_SMEM_MAX));
-        attr_done = true;
+        if (attr_done) *attr_done = true;
     }
     MTV_CUDA_CHECK(cudaMemsetAsync(keys, 0, (size_t)M * 8, st));
     int ctas = sm_count() / passes;                      // per pass; one CTA per SM in all

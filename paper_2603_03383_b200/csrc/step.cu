@@ -1,4 +1,6 @@
 // Whole verification step on one stream, and its host-buffer variant.
+#include <mutex>
+
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -50,16 +52,23 @@ extern "C" int mtv_verify_step(const mtv_tree_t *tree, const mtv_step_args *a, v
 }
 
 namespace {
-// Copy streams and events of the host-buffer variant, created on first use (one set per process;
-// the variant synchronises anyway, so it is not one of the allocation-free hot calls).
+// Copy streams and events of the host-buffer variant, created on first use, one set per device (the variant
+// synchronises anyway, so it is not one of the allocation-free hot calls).  Calls on one device take turns.
 struct HostStepAux {
     cudaStream_t up = nullptr, down = nullptr;
     cudaEvent_t start = nullptr, q_up = nullptr, logits_up = nullptr, down_done = nullptr;
     cudaEvent_t chunk[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     bool ready = false;
+    std::mutex busy;
 };
-HostStepAux g_aux;
-int host_step_aux() {
+HostStepAux g_aux_table[mtv::MTV_MAX_DEVICES];
+int host_step_aux(HostStepAux **out) {
+    int dev = 0;
+    MTV_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= mtv::MTV_MAX_DEVICES) return MTV_ERR_UNSUPPORTED_SHAPE;
+    HostStepAux &g_aux = g_aux_table[dev];
+    *out = &g_aux;
+    std::lock_guard<std::mutex> lock(g_aux.busy);
     if (g_aux.ready) return MTV_OK;
     MTV_CUDA_CHECK(cudaStreamCreateWithFlags(&g_aux.up, cudaStreamNonBlocking));
     MTV_CUDA_CHECK(cudaStreamCreateWithFlags(&g_aux.down, cudaStreamNonBlocking));
@@ -77,7 +86,10 @@ int host_step_aux() {
 extern "C" int mtv_verify_step_host(const mtv_tree_t *tree, const mtv_step_args *d, const mtv_step_args *h,
                                     void *stream) {
     if (!tree || !d || !h || !d->k_caches_host || !d->v_caches_host) return MTV_ERR_INVALID_ARG;
-    if (host_step_aux() != MTV_OK) return MTV_ERR_CUDA;
+    HostStepAux *aux = nullptr;
+    if (host_step_aux(&aux) != MTV_OK) return MTV_ERR_CUDA;
+    HostStepAux &g_aux = *aux;
+    std::lock_guard<std::mutex> turn(g_aux.busy);
     cudaStream_t st = (cudaStream_t)stream, up = g_aux.up, down = g_aux.down;
     const size_t B = d->B, T = tree->T, K = tree->K;
     const size_t per_layer = B * T * d->Hq * d->D;           // elements

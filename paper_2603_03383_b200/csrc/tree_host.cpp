@@ -31,14 +31,14 @@ void set_last_error(const char *what, cudaError_t e) {
 }
 void set_last_error_text(const char *text) { snprintf(g_err, sizeof g_err, "%s", text); }
 int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-            n = 148;
+    static int n[MTV_MAX_DEVICES] = {0};
+    int dev = 0, count = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MTV_MAX_DEVICES) return 148;
+    if (n[dev] == 0) {
+        if (cudaDeviceGetAttribute(&count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || count <= 0) count = 148;
+        n[dev] = count;
     }
-    return n;
+    return n[dev];
 }
 Tap g_taps[MTV_KERNEL_COUNT];
 }  // namespace mtv

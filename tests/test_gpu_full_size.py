@@ -1,7 +1,7 @@
 """GPU parity at the full sizes of the five benchmark configurations, in the launch configuration
-that bench.py times.  The checker cannot compute every output at these sizes in seconds, so
-attention is compared on sampled (sequence, node, head) rows; integer outputs are compared in full
-(top-k ids for sampled batch rows, acceptance for every sequence)."""
+that bench.py times.  Attention is compared on every row where the checker finishes in seconds, else on rows
+that cover every sequence, KV head and row tile; integer outputs are compared in full (top-k ids for sampled
+batch rows, acceptance for every sequence)."""
 import pytest
 import torch
 
@@ -13,16 +13,27 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-def _sample_rows(B, T, Hq, n, seed):
+def _covering_rows(B, T, Hq, Hkv, per_cell, seed):
+    """(sequence, node, head) rows that reach every (sequence, KV head, 128-row tile of the (node, head-in-group)
+    block) at least `per_cell` times, plus the corners."""
+    G = Hq // Hkv
+    tiles = (T * G + 127) // 128
     g = torch.Generator().manual_seed(seed)
-    rows = torch.stack([torch.randint(0, B, (n,), generator=g), torch.randint(0, T, (n,), generator=g),
-                        torch.randint(0, Hq, (n,), generator=g)], dim=1).tolist()
+    rows = []
+    for b in range(B):
+        for kv in range(Hkv):
+            for t in range(tiles):
+                lo, hi = t * 128, min(T * G, t * 128 + 128)
+                for r in torch.randint(lo, hi, (per_cell,), generator=g).tolist():
+                    rows.append([b, r // G, kv * G + r % G])
     rows += [[0, 0, 0], [B - 1, T - 1, Hq - 1], [0, T - 1, 0], [B - 1, 0, Hq - 1]]     # root and last node, first and last head
     return rows
 
 
-@pytest.mark.parametrize("name,n_rows", [("tiny", 64), ("short", 96), ("long", 96), ("batched", 160), ("stress", 64)])
-def test_attention_full_size_sampled_rows(name, n_rows):
+@pytest.mark.parametrize("name,per_cell", [("tiny", 0), ("short", 0), ("long", 0), ("batched", 2), ("stress", 4)])
+def test_attention_full_size(name, per_cell):
+    """Every output row at `tiny`, `short` and `long`; at `batched` and `stress` (where the checker would take minutes)
+    at least 512 rows that reach every sequence, KV head and row tile."""
     w = synth.WORKLOADS[name]
     tb, tree = workload_tree(w)
     T, B = tree.T, w.B
@@ -36,11 +47,16 @@ def test_attention_full_size_sampled_rows(name, n_rows):
     torch.cuda.synchronize()
     assert status.tolist() == [0] * B
     assert binding.mtv_device_error(tree) == 0
-    rows = _sample_rows(B, T, w.Hq, n_rows, w.cfg_id)
-    want = ref.tree_attention(q.cpu(), k.cpu(), v.cpu(), lens, tb["mask"], rows=rows)
-    idx = torch.tensor(rows)
-    got = out.cpu()[idx[:, 0], idx[:, 1], idx[:, 2]]
-    assert_close(got, want, "%s attention, sampled rows" % name)
+    if per_cell == 0:
+        want = ref.tree_attention(q.cpu(), k.cpu(), v.cpu(), lens, tb["mask"])
+        assert_close(out, want, "%s attention, every row" % name)
+    else:
+        rows = _covering_rows(B, T, w.Hq, w.Hkv, per_cell, w.cfg_id)
+        assert len(rows) >= 512
+        want = ref.tree_attention(q.cpu(), k.cpu(), v.cpu(), lens, tb["mask"], rows=rows)
+        idx = torch.tensor(rows)
+        got = out.cpu()[idx[:, 0], idx[:, 1], idx[:, 2]]
+        assert_close(got, want, "%s attention, %d rows" % (name, len(rows)))
     # a property that holds for every row: each output is a convex combination of V rows
     vmax = v.float().abs().max().item()
     assert out.float().abs().max().item() <= vmax * 1.01 and bool(torch.isfinite(out.float()).all())
@@ -99,7 +115,7 @@ def test_accept_full_size(name):
 
 @pytest.mark.parametrize("name,reps", [("long", 300), ("short", 300), ("stress", 20)])
 def test_attention_is_bitwise_repeatable(name, reps):
-    """The key splits of a query block meet through counters and bulk copies inside one launch; the merge order
+    """The key splits of a query block meet through counters and the workspace inside one launch; the merge order
     is fixed, so repeated calls must give bit-identical output.  A missing fence in that exchange would show up
     here as a rare difference."""
     w = synth.WORKLOADS[name]

@@ -114,13 +114,19 @@ def test_accept_from_lm_head_keys():
         assert torch.equal(t.cpu(), want[name]), name
 
 
-def test_lm_head_full_size_7b():
-    """The configuration the step benchmark runs: 64 nodes, H = 4096, V = 32000."""
+@pytest.mark.parametrize("V", [32000, 131072])
+def test_lm_head_full_size_7b(V):
+    """64 nodes, H = 4096; V = 131072 is the vocabulary the step benchmark runs, V = 32000 one whose tiling has a
+    ragged last slab."""
     tb, tree = make_tree("rank_prior", 4, (), 64)
-    H, V = 4096, 32000
+    H = 4096
     x = synth.normal_bf16(14, 1, (1, tree.T, H))
     W = synth.normal_bf16(14, 2, (V, H), scale=0.02)
     keys, am, val = _run(tree, x, W)
-    _check(x, W, am, val)
+    if V > 100000:      # the checker on every fourth node (its fp64 product over the whole vocabulary takes a second per node)
+        sel = torch.arange(0, tree.T, 4)
+        _check(x[:, sel], W, am[sel], val[sel])
+    else:
+        _check(x, W, am, val)
     keys2, am2, val2 = _run(tree, x, W)
     assert torch.equal(keys, keys2)                          # bitwise repeatable

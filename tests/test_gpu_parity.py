@@ -359,6 +359,109 @@ def test_full_step_with_fused_lm_head_from_host_buffers():
     _step_case(2, 256, 2000, 8, 2, 64, 2, "cartesian", 3, (4, 2, 2), 0, [90, 33], seed=8, host=True, lm_head=True)
 
 
+def test_full_step_at_the_long_shapes():
+    """Hidden size, vocabulary, heads and prefix of the `long` configuration (two layers: the checker's attention
+    takes seconds per layer), every output and the compacted caches against the checker."""
+    w = synth.WORKLOADS["long"]
+    _step_case(w.B, w.H, w.V, w.Hq, w.Hkv, w.D, 2, w.tree, w.K, w.topk, w.T, [w.L_lo], w.seed)
+
+
+def test_full_step_from_host_buffers_with_more_layers_than_download_groups():
+    """Twenty layers: the attention outputs leave in groups of two layers (sixteen groups at most)."""
+    _step_case(2, 256, 2000, 8, 2, 128, 20, "rank_prior", 4, (), 64, [70, 33], seed=9, host=True)
+
+
+def test_three_chained_steps():
+    """Step, compaction, append of the next tree's K/V with the rotary embedding, step again: attention of a later
+    step reads the cache that this library's own compaction and append produced, and the whole chain equals the
+    checker stepping the same way (the accepted path's K/V are what sequential decoding would have appended)."""
+    B, H, V, Hq, Hkv, D, K, n_layers = 2, 256, 2000, 8, 2, 128, 4, 2
+    tb, tree = make_tree("rank_prior", K, (), 64)
+    T = tree.T
+    lens0 = [150, 37]
+    Lcap = max(lens0) + 3 * (K + 1) + T
+    seed = 77
+    f = lambda *s_: torch.full(s_, -7, dtype=torch.int32, device=DEV)
+    # state: caches and lengths, on both sides
+    kc = [synth.normal_bf16(seed, 500 + l, (B, Hkv, Lcap, D)) for l in range(n_layers)]
+    vc = [synth.normal_bf16(seed, 600 + l, (B, Hkv, Lcap, D)) for l in range(n_layers)]
+    kd, vd = [t.to(DEV) for t in kc], [t.to(DEV) for t in vc]
+    sl_ref = torch.tensor(lens0, dtype=torch.int32)
+    sl_dev = sl_ref.to(DEV)
+    root_ref = synth.uniform_int(seed, 7, B, 0, V - 1).to(torch.int32)
+    root_dev = root_ref.to(DEV)
+    ws = workspace(tree, B, H, V, Hq, Hkv, D, Lcap)
+    kp, vp = binding.cache_pointer_array(kd, DEV), binding.cache_pointer_array(vd, DEV)
+    strides = (Hkv * Lcap * D, Lcap * D, D)
+    for step in range(3):
+        # ---- inputs of this step (same values on both sides); the heads' seed is bumped until the checker's rank
+        #      gaps clear the margin
+        s_in = seed + 10 * step
+        for attempt in range(20):
+            hidden, W1, b1, W2, _ = synth.head_inputs(B, H, V, K, s_in)
+            z = ref.heads_logits(hidden, W1, b1, W2)
+            cand_ref, _, tt_ref, gap = ref.heads_candidates(z, root_ref, tb)
+            if gap > 1e-5 * z.abs().max().item():
+                break
+            s_in += 1000
+        q = [synth.normal_bf16(s_in, 700 + l, (B, T, Hq, D)) for l in range(n_layers)]
+        kn = [synth.normal_bf16(s_in, 800 + l, (B, T, Hkv, D)) for l in range(n_layers)]
+        vn = [synth.normal_bf16(s_in, 900 + l, (B, T, Hkv, D)) for l in range(n_layers)]
+        logits, planted = synth.planted_logits(B, T, V, K, tt_ref, tb["parent"], tb["rank"], s_in, p_accept=(0.9, 0.6))
+        # ---- the checker's step
+        out_ref = []
+        for l in range(n_layers):
+            q_rot, k_rot = ref.rope(q[l], kn[l], sl_ref.tolist(), tb["depth"])
+            for b in range(B):
+                L = int(sl_ref[b])
+                kc[l][b, :, L:L + T] = k_rot[b].to(torch.bfloat16).permute(1, 0, 2)
+                vc[l][b, :, L:L + T] = vn[l][b].permute(1, 0, 2)
+            out_ref.append(ref.tree_attention(q_rot.to(torch.bfloat16), kc[l], vc[l], sl_ref, tb["mask"]))
+        acc_ref = ref.tree_accept(ref.node_argmax(logits), tt_ref, tb)
+        assert torch.equal(acc_ref["accept_len"], planted)
+        new_len = None
+        for l in range(n_layers):
+            kc[l], new_len = ref.kv_compact(kc[l], sl_ref, acc_ref["accept_len"], acc_ref["acc_nodes"])
+            vc[l], _ = ref.kv_compact(vc[l], sl_ref, acc_ref["accept_len"], acc_ref["acc_nodes"])
+        # ---- this library's step, call by call
+        cand, tt = f(B, tree.C), f(B, T)
+        binding.medusa_heads_topk(tree, hidden.to(DEV), W1.to(DEV), b1.to(DEV), W2.to(DEV), root_dev, cand, None, tt, ws)
+        assert torch.equal(tt.cpu(), tt_ref) and torch.equal(cand.cpu(), cand_ref)
+        status = f(B)
+        for l in range(n_layers):
+            qd = q[l].to(DEV)
+            binding.tree_kv_append_rope(tree, qd, kn[l].to(DEV), vn[l].to(DEV), kd[l], vd[l], sl_dev, status=status)
+            out = torch.zeros(B, T, Hq, D, dtype=torch.bfloat16, device=DEV)
+            binding.tree_verify_attention(tree, qd, kd[l], vd[l], sl_dev, out, ws, status=status)
+            torch.cuda.synchronize()
+            assert status.tolist() == [0] * B
+            assert_close(out, out_ref[l], "step %d layer %d" % (step, l))
+        outs = dict(accept_len=f(B), best_path=f(B), acc_nodes=f(B, K + 1), acc_tok=f(B, K + 1), next_root=f(B))
+        binding.tree_accept(tree, logits.to(DEV), tt, outs["accept_len"], outs["best_path"], outs["acc_nodes"],
+                            outs["acc_tok"], outs["next_root"], ws)
+        binding.kv_compact_accepted(tree, kp, vp, n_layers, B, Hkv, D, strides, Lcap, sl_dev, outs["accept_len"],
+                                    outs["acc_nodes"], status=status)
+        torch.cuda.synchronize()
+        for name, t in outs.items():
+            assert torch.equal(t.cpu(), acc_ref[name]), (step, name)
+        assert status.tolist() == [0] * B and torch.equal(sl_dev.cpu(), new_len)
+        for l in range(n_layers):
+            for b in range(B):
+                # V rows are copies: bit-exact.  The appended K rows were rotated in fp32 here and in fp64 by the
+                # checker before the rounding to bf16: equal to the float tolerance, and bit-exact below the first
+                # appended row
+                n, n0 = int(new_len[b]), lens0[b]
+                assert torch.equal(vd[l][b, :, :n].cpu(), vc[l][b, :, :n])
+                assert torch.equal(kd[l][b, :, :n0].cpu(), kc[l][b, :, :n0])
+                assert_close(kd[l][b, :, :n], kc[l][b, :, :n], "compacted K rows")
+        # ---- the next step starts from the token after the accepted path
+        sl_ref = new_len
+        root_ref = acc_ref["next_root"]
+        root_dev = outs["next_root"]
+    assert binding.mtv_device_error(tree) == 0
+    assert int(sl_ref.min()) > min(lens0)
+
+
 def test_generator_is_identical_on_cpu_and_gpu():
     a = synth.normal_bf16(123, 5, (1 << 16,), 0.37)
     b = synth.normal_bf16(123, 5, (1 << 16,), 0.37, device=DEV)
