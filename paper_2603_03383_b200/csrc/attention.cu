@@ -20,7 +20,7 @@ bool attn_tc_eligible(int D, int G);
 int attn_tc_plan(int T, int G, int B, int Hkv, int Lcap, int *n_rt_out);
 int launch_tree_attn_tc(const mtv_tree *tree, int B, int Hq, int Hkv, const __nv_bfloat16 *q, const __nv_bfloat16 *k,
                         const __nv_bfloat16 *v, int64_t sb, int64_t sh, int64_t st, int Lcap, const int32_t *seq_lens,
-                        float scale_log2, __nv_bfloat16 *out, int32_t *status, void *ws_o, float *ws_ml,
+                        float scale_log2, __nv_bfloat16 *out, int32_t *status, void *ws_o, float *ws_ml, int32_t *ws_order,
                         cudaStream_t stream);
 
 AttnWs attn_ws_layout(const mtv_tree *t, int B, int Hq, int Hkv, int D, int Lcap) {
@@ -35,7 +35,8 @@ AttnWs attn_ws_layout(const mtv_tree *t, int B, int Hq, int Hkv, int D, int Lcap
         const size_t slabs = w.nsplit > 1 ? (size_t)B * Hkv * n_rt * w.nsplit : 0;
         w.o_off = 0;
         w.ml_off = align_up(slabs * 256 * D * sizeof(__nv_bfloat16), 256);
-        w.total = align_up(w.ml_off + slabs * 256 * 2 * sizeof(float), 256) + 256;
+        w.order_off = align_up(w.ml_off + slabs * 256 * 2 * sizeof(float), 256);   // sequences by descending length
+        w.total = align_up(w.order_off + (size_t)B * sizeof(int32_t), 256) + 256;
         return w;
     }
     const int mblocks = (M + BM - 1) / BM;
@@ -339,7 +340,8 @@ extern "C" int tree_verify_attention(const mtv_tree_t *tree, int B, int Hq, int 
         // tcgen05 path: head_dim 128, query groups of 1/2/4/8 heads; one launch
         TapScope tap(MTV_KERNEL_ATTN_PARTIAL, st);
         const int rc = launch_tree_attn_tc(tree, B, Hq, Hkv, p.q, p.k, p.v, stride_b, stride_h, stride_t, Lcap, seq_lens,
-                                           p.scale_log2, p.out, status, p.ws_o, p.ws_ml, st);
+                                           p.scale_log2, p.out, status, p.ws_o, p.ws_ml,
+                                           reinterpret_cast<int32_t *>((char *)ws + Lw.order_off), st);
         if (rc != MTV_OK) return rc;
         MTV_CUDA_CHECK(cudaGetLastError());
         return MTV_OK;

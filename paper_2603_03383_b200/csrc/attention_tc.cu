@@ -110,6 +110,7 @@ struct TcParams {
     float2 *ws_ml;         // [query blocks][nsplit][256] partial (m, l)
     int32_t *arrive, *depart;   // [query blocks][2] merge counters, zero between calls
     int32_t *status;       // [B] or null
+    const int32_t *order;  // [B] sequences by descending length, or null: grid index z -> sequence
     int32_t *dev_error;
     float scale_log2;
     int T, G, Hq, Hkv, Lcap, nsplit, n_blk, M_rows;
@@ -188,7 +189,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     const uint32_t rank = ptx::cluster_ctarank();     // 0: issues the MMAs, rows 0-127 of the block; 1: rows 128-255
     const int split = blockIdx.x >> 1;
     const int g = blockIdx.y / p.n_blk, blk = blockIdx.y % p.n_blk;
-    const int b = blockIdx.z;
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     TRACE_INIT;
     if (warp == 0) TRACE(0);
@@ -246,6 +246,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     // Nothing above touched global memory.  From here on the previous kernel of the stream must be
     // complete (its outputs may be this kernel's inputs, and it may share the workspace and counters).
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // With more query blocks than CTA pairs fit the device, blocks start in grid order as pairs retire: the longest
+    // sequences go first (the order comes from a small kernel in front of this one), so that the last pairs to start
+    // are the shortest.
+    const int b = p.order ? p.order[blockIdx.z] : blockIdx.z;
     const int L = p.seq_lens[b];
     const int rows0 = blk * 256 + (int)rank * 128;   // first row of this CTA inside the (sequence, KV head) block
     auto tile_of = [&](int j) { return split + j * p.nsplit; };
@@ -807,6 +811,21 @@ static bool encode_map(CUtensorMap *map, const void *base, const cuuint64_t dims
     return true;
 }
 
+// order[r] = the sequence with the r-th largest length (ties: lower index first).  B is small: every thread ranks one
+// sequence against all others.
+__global__ void attn_order_kernel(const int32_t *seq_lens, int B, int32_t *order) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const int len = seq_lens[b];
+    int rank = 0;
+    for (int o = 0; o < B; ++o) {
+        const int lo = seq_lens[o];
+        rank += (lo > len || (lo == len && o < b)) ? 1 : 0;
+    }
+    order[rank] = b;
+}
+constexpr int TC_ORDER_MAX_B = 2048;
+
 bool attn_tc_eligible(int D, int G) { return D == 128 && (G == 1 || G == 2 || G == 4 || G == 8); }
 
 static int tc_prepare() {
@@ -836,7 +855,7 @@ int attn_tc_plan(int T, int G, int B, int Hkv, int Lcap, int *n_blk_out) {
 
 int launch_tree_attn_tc(const mtv_tree *tree, int B, int Hq, int Hkv, const __nv_bfloat16 *q, const __nv_bfloat16 *k,
                         const __nv_bfloat16 *v, int64_t sb, int64_t sh, int64_t st, int Lcap, const int32_t *seq_lens,
-                        float scale_log2, __nv_bfloat16 *out, int32_t *status, void *ws_o, float *ws_ml,
+                        float scale_log2, __nv_bfloat16 *out, int32_t *status, void *ws_o, float *ws_ml, int32_t *ws_order,
                         cudaStream_t stream) {
     const int G = Hq / Hkv, T = tree->T, D = 128;
     CUtensorMap q_map, k_map, v_map;
@@ -861,6 +880,11 @@ int launch_tree_attn_tc(const mtv_tree *tree, int B, int Hq, int Hkv, const __nv
     p.T = T; p.G = G; p.Hq = Hq; p.Hkv = Hkv; p.Lcap = Lcap;
     p.nsplit = attn_tc_plan(T, G, B, Hkv, Lcap, &p.n_blk);
     p.M_rows = T * G;
+    p.order = nullptr;
+    if (p.nsplit == 1 && B > 1 && B <= TC_ORDER_MAX_B && (long)B * Hkv * p.n_blk > sm_count() / 2 && ws_order) {
+        attn_order_kernel<<<(B + 255) / 256, 256, 0, stream>>>(seq_lens, B, ws_order);
+        p.order = ws_order;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * p.nsplit, Hkv * p.n_blk, B);   // the kernel's cluster is (2, 1, 1): a CTA pair
     cfg.blockDim = dim3(TC_THREADS, 1, 1);

@@ -60,7 +60,7 @@ int launch_heads_tc(const mtv_tree *t, int B, int H, int V, const __nv_bfloat16 
                     float *cand_logit, int32_t *tree_tok, const HeadsWs &L, char *ws, cudaStream_t st);
 
 struct AttnWs {
-    size_t o_off, ml_off, total;
+    size_t o_off, ml_off, order_off = 0, total;
     int nsplit, m_rows;
     bool use_tc;   // head_dim 128 path on the tcgen05 tensor cores
 };
