@@ -52,6 +52,9 @@ extern "C" {
 #define MTV_ERR_CUDA (-4)
 #define MTV_ERR_TIMEOUT (-5)
 #define MTV_ERR_CAPACITY (-6) /* status[b]: seq_lens[b] + T exceeds the cache capacity */
+#define MTV_ERR_BOUNDS (-7)   /* device error word, -DMTV_DEBUG_BOUNDS builds only: an index read from device
+                                 memory (a tree table, acc_nodes, accept_len, the sequence order) was out of
+                                 range; the access was skipped */
 
 #define MTV_MAX_K 8
 #define MTV_MAX_T 128
@@ -153,6 +156,15 @@ int tree_kv_append_rope(const mtv_tree_t *tree, int B, int Hq, int Hkv, int D, m
                         int64_t stride_b, int64_t stride_h, int64_t stride_t, int Lcap,
                         const int32_t *seq_lens, float rope_theta, int32_t *status, void *stream);
 
+/* The same for all n_layers caches of a step in one launch: q_layers [n_layers][B][T][Hq][D] (rotated
+ * in place), k_new_layers, v_new_layers [n_layers][B][T][Hkv][D]; k_caches / v_caches: device arrays of
+ * n_layers device pointers, as for kv_compact_accepted. */
+int tree_kv_append_rope_layers(const mtv_tree_t *tree, int B, int Hq, int Hkv, int D, int n_layers,
+                               mtv_bf16 *q_layers, const mtv_bf16 *k_new_layers, const mtv_bf16 *v_new_layers,
+                               mtv_bf16 *const *k_caches, mtv_bf16 *const *v_caches,
+                               int64_t stride_b, int64_t stride_h, int64_t stride_t, int Lcap,
+                               const int32_t *seq_lens, float rope_theta, int32_t *status, void *stream);
+
 /* ---------------------------------------------------------------------------
  * Tree attention — Section 3.2 / Fig. 2(b): the T tree nodes attend to the KV cache
  * under the static visibility matrix.  For sequence b, node i, query head h
@@ -165,6 +177,19 @@ int tree_kv_append_rope(const mtv_tree_t *tree, int B, int Hq, int Hkv, int D, m
  * multiples of 8; base 16-byte aligned); the caller has already written the tree
  * nodes' K/V to rows seq_lens[b] + i.  seq_lens [B] device int32 (0 is legal).
  * scale == 0 means 1/sqrt(D).  status[b] = MTV_ERR_CAPACITY if seq_lens[b] + T > Lcap.
+ * Precondition at head size 128 when one sequence's keys are split over several thread-block
+ * pairs (few, long sequences: B * Hkv * ceil(T*Hq/Hkv / 256) at most half the pairs the device
+ * holds): the splits of a query block meet inside the launch through counters in the workspace,
+ * so all blocks of the launch must be resident at once.  The grid is sized to fit an idle
+ * device (one block per SM); do not run the call while another long-running kernel occupies
+ * SMs of the same device (other streams, other processes under MPS).  If the blocks cannot
+ * meet, the bounded waits run out after about a second, the tree's device error word reads
+ * MTV_ERR_TIMEOUT and the output is undefined — the call never hangs.  Calls that share a
+ * tree or a workspace must not overlap on the device.  The encoded tensor maps of (pointer,
+ * shape, strides) are kept in a process-wide table; a mutex guards it, so calls from several
+ * host threads are safe.
+ * Development build option -DMTV_TRACE: the head-size-128 kernel stamps the cycle counter at
+ * its phases into a buffer given by mtv_trace_set (absent from normal builds).
  */
 int tree_verify_attention(const mtv_tree_t *tree, int B, int Hq, int Hkv, int D,
                           const mtv_bf16 *q, const mtv_bf16 *k_cache, const mtv_bf16 *v_cache,
@@ -182,8 +207,12 @@ int tree_verify_attention(const mtv_tree_t *tree, int B, int Hq, int Hkv, int D,
  *   best_path = argmax_p len_p (ties: lowest p);  accept_len = len_best in [0, K]
  *   acc_nodes[b][0..accept_len] = ri[best][..], acc_tok = tree_tok at those nodes, -1 padded
  *   next_root[b] = am[b][acc_nodes[b][accept_len]]
- * All pointers device.  logits [B][T][V] bf16 (base-model logits at every tree node).
+ * All pointers device.  logits [B][T][V] bf16 (base-model logits at every tree node), base
+ * address 16-byte aligned (rows are scanned in 16-byte chunks; a misaligned base is refused
+ * with MTV_ERR_INVALID_ARG and nothing is launched; V need not be a multiple of 8).
  * Outputs: accept_len, best_path, next_root [B]; acc_nodes, acc_tok [B][K+1].
+ * Host threads: the per-device launch set-up is remembered in plain flags; two threads that
+ * make their first call on a device at the same time both do the (idempotent) set-up.
  */
 int tree_accept(const mtv_tree_t *tree, int B, int V, const mtv_bf16 *logits, const int32_t *tree_tok,
                 int32_t *accept_len, int32_t *best_path, int32_t *acc_nodes, int32_t *acc_tok,
@@ -290,6 +319,33 @@ typedef struct {
 
 int mtv_verify_step(const mtv_tree_t *tree, const mtv_step_args *args, void *stream);
 
+/* ---------------------------------------------------------------------------
+ * A chain of n_steps verification steps enqueued on one stream with no host decision between
+ * them — Section 3.2: the step is one static graph without dynamic control flow, and nothing
+ * the next step needs (the accepted length, the compacted cache, the next root token) passes
+ * through the CPU.  steps[s] describes step s as for mtv_verify_step; within a chain
+ *   - steps[s].root_tok == NULL (s >= 1) means "the previous step's next_root" (device pointer
+ *     steps[s-1].next_root, read when step s runs);
+ *   - all steps share one seq_lens array, advanced on the device by every step's compaction.
+ * appends (NULL, or n_steps entries): where appends[s].k_new_layers / v_new_layers are given,
+ * step s first writes its tree nodes' K/V rows into the caches — all layers in one launch of
+ * tree_kv_append_rope's kernel, directly in front of the step's first attention call, which
+ * starts its set-up under that kernel's tail (programmatic dependent launch) — and rotates
+ * steps[s].q_layers in place (so that buffer must be writable although the struct says const).
+ * k_new_layers, v_new_layers: [n_layers][B][T][Hkv][D] device, un-rotated K rows and V rows;
+ * rope_theta == 0 means 10000.  Per-step inputs that a backbone would compute from the previous
+ * step's tokens (hidden, q, k_new, v_new, logits / x_final) are the caller's, laid out per step
+ * before the call: the backbone is outside this library.
+ * Errors: as the calls it chains; MTV_ERR_INVALID_ARG for a first step without root_tok or
+ * steps that name different seq_lens.  Nothing is rolled back when a later step is refused. */
+typedef struct {
+    const mtv_bf16 *k_new_layers, *v_new_layers;
+    float rope_theta;
+} mtv_append_args;
+
+int mtv_verify_steps(const mtv_tree_t *tree, const mtv_step_args *steps, const mtv_append_args *appends,
+                     int n_steps, void *stream);
+
 /* The same step for a caller whose per-step tensors live in (pinned) host memory.
  * Copies hidden, root_tok, q_layers and logits host->device into the device
  * buffers named in `dev`, runs the step, copies tree_tok, out_layers,
@@ -342,6 +398,13 @@ int mtv_device_error(const mtv_tree_t *tree, int clear, int32_t *code);
  * tree's device error word and returns normally: nothing faults, the context stays usable.
  * Only enqueues the kernel; read the word with mtv_device_error afterwards. */
 int mtv_selftest_wait_timeout(const mtv_tree_t *tree, void *stream);
+
+/* 1 if the library was compiled with -DMTV_DEBUG_BOUNDS, else 0 (the paper has no counterpart).  That build
+ * checks every index that a kernel reads from device memory before it is used as an address — tree tables,
+ * acc_nodes / accept_len handed to the compaction, the length-ranked sequence order — records MTV_ERR_BOUNDS in the
+ * tree's device error word and skips the access instead of following it: a stand-in for a memory checker
+ * where none can be run.  Results are otherwise identical; the checks cost a few instructions per index. */
+int mtv_debug_bounds_enabled(void);
 
 /* Human-readable text for the most recent MTV_ERR_CUDA (or refused size) on this thread (never NULL). */
 const char *mtv_last_error(void);

@@ -14,10 +14,12 @@ from typing import Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmtv.so")
+# MTV_LIB names another build of the same library (a variant of build.py, e.g. the bounds-checking one).
+LIB_PATH = os.environ.get("MTV_LIB") or os.path.join(_HERE, "libmtv.so")
 
 MTV_OK = 0
-ERR = {-1: "MTV_ERR_INVALID_ARG", -2: "MTV_ERR_UNSUPPORTED_SHAPE", -3: "MTV_ERR_WORKSPACE",
+MTV_ERR_BOUNDS = -7
+ERR = {-7: "MTV_ERR_BOUNDS", -1: "MTV_ERR_INVALID_ARG", -2: "MTV_ERR_UNSUPPORTED_SHAPE", -3: "MTV_ERR_WORKSPACE",
        -4: "MTV_ERR_CUDA", -5: "MTV_ERR_TIMEOUT", -6: "MTV_ERR_CAPACITY"}
 MTV_ERR_TIMEOUT = -5
 MTV_ERR_CAPACITY = -6
@@ -28,7 +30,8 @@ EXPORTS = ["tree_build_static", "tree_gen_cartesian", "tree_gen_rank_prior", "tr
            "kv_compact_accepted", "mtv_verify_step", "mtv_verify_step_host", "mtv_last_error",
            "mtv_set_kernel_taps", "mtv_kernel_taps_used", "mtv_device_error",
            "tree_accept_static_scratch", "tree_accept_static_scratch_capacity", "tree_kv_append_rope",
-           "lm_head_argmax", "tree_accept_keys", "mtv_selftest_wait_timeout"]
+           "lm_head_argmax", "tree_accept_keys", "mtv_selftest_wait_timeout", "tree_kv_append_rope_layers",
+           "mtv_verify_steps", "mtv_debug_bounds_enabled"]
 
 
 class MtvError(RuntimeError):
@@ -66,6 +69,10 @@ class StepArgs(C.Structure):
                 ("acc_tok", C.c_void_p), ("next_root", C.c_void_p), ("status", C.c_void_p),
                 ("ws", C.c_void_p), ("ws_bytes", C.c_size_t),
                 ("x_final", C.c_void_p), ("W_lm", C.c_void_p)]
+
+
+class AppendArgs(C.Structure):
+    _fields_ = [("k_new_layers", C.c_void_p), ("v_new_layers", C.c_void_p), ("rope_theta", C.c_float)]
 
 
 _lib = None
@@ -106,6 +113,9 @@ def lib():
         L.lm_head_argmax.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         L.tree_accept_keys.argtypes = [vp, i32] + [vp] * 7 + [vp]
         L.mtv_selftest_wait_timeout.argtypes = [vp, vp]
+        L.tree_kv_append_rope_layers.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, i64, i64, i64, i32, vp,
+                                                 C.c_float, vp, vp]
+        L.mtv_verify_steps.argtypes = [vp, C.POINTER(StepArgs), C.POINTER(AppendArgs), i32, vp]
         _lib = L
     return _lib
 
@@ -187,6 +197,10 @@ def mtv_device_error(tree: Tree, clear: bool = True) -> int:
     return code.value
 
 
+def mtv_debug_bounds_enabled() -> bool:
+    return bool(lib().mtv_debug_bounds_enabled())
+
+
 def mtv_selftest_wait_timeout(tree: Tree, stream=None):
     """Enqueue a kernel whose bounded wait must run out (about a second); see include/mtv.h."""
     _check(lib().mtv_selftest_wait_timeout(tree.handle, _stream(stream)), "mtv_selftest_wait_timeout")
@@ -232,6 +246,19 @@ def tree_kv_append_rope(tree, q, k_new, v_new, k_cache, v_cache, seq_lens, rope_
     _check(lib().tree_kv_append_rope(tree.handle, B, Hq, Hkv, D, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache),
                                      _ptr(v_cache), sb, sh, st, Lcap, _ptr(seq_lens), rope_theta, _ptr(status),
                                      _stream(stream)), "tree_kv_append_rope")
+
+
+def tree_kv_append_rope_layers(tree, q_layers, k_new_layers, v_new_layers, k_ptrs, v_ptrs, strides, Lcap, seq_lens,
+                               rope_theta=0.0, status=None, stream=None):
+    """q_layers [n_layers][B][T][Hq][D], k_new_layers / v_new_layers [n_layers][B][T][Hkv][D]; k_ptrs / v_ptrs as for
+    kv_compact_accepted."""
+    n_layers, B, T, Hq, D = q_layers.shape
+    Hkv = k_new_layers.shape[3]
+    sb, sh, st = strides
+    _check(lib().tree_kv_append_rope_layers(tree.handle, B, Hq, Hkv, D, n_layers, _ptr(q_layers), _ptr(k_new_layers),
+                                            _ptr(v_new_layers), _ptr(k_ptrs), _ptr(v_ptrs), sb, sh, st, Lcap,
+                                            _ptr(seq_lens), rope_theta, _ptr(status), _stream(stream)),
+           "tree_kv_append_rope_layers")
 
 
 def tree_accept(tree, logits, tree_tok, accept_len, best_path, acc_nodes, acc_tok, next_root, ws, stream=None):
@@ -287,6 +314,17 @@ def kv_compact_accepted(tree, k_ptrs, v_ptrs, n_layers, B, Hkv, D, strides, Lcap
 
 def mtv_verify_step(tree, args: StepArgs, stream=None):
     _check(lib().mtv_verify_step(tree.handle, C.byref(args), _stream(stream)), "mtv_verify_step")
+
+
+def mtv_verify_steps(tree, steps: Sequence[StepArgs], appends: Optional[Sequence[AppendArgs]] = None, stream=None):
+    """A chain of steps on one stream (see include/mtv.h); `steps` and `appends` are sequences of the structs."""
+    n = len(steps)
+    arr = (StepArgs * n)(*steps)
+    app = None
+    if appends is not None:
+        assert len(appends) == n
+        app = (AppendArgs * n)(*appends)
+    _check(lib().mtv_verify_steps(tree.handle, arr, app, n, _stream(stream)), "mtv_verify_steps")
 
 
 def mtv_verify_step_host(tree, dev: StepArgs, host: StepArgs, stream=None):

@@ -104,7 +104,7 @@ accept_finish_kernel(int T, int K, int P, int ns, const unsigned long long *__re
                      const int32_t *__restrict__ tree_tok, const int32_t *__restrict__ ri,
                      int32_t *__restrict__ accept_len, int32_t *__restrict__ best_path,
                      int32_t *__restrict__ acc_nodes, int32_t *__restrict__ acc_tok,
-                     int32_t *__restrict__ next_root) {
+                     int32_t *__restrict__ next_root, int32_t *__restrict__ dev_error) {
     __shared__ int32_t am[MTV_MAX_T];
     __shared__ int32_t tok[MTV_MAX_T];
     __shared__ unsigned int best_key;
@@ -123,7 +123,9 @@ accept_finish_kernel(int T, int K, int P, int ns, const unsigned long long *__re
         int len = 0;
         for (int j = 1; j <= K; ++j) {
             const int node = path[j];
-            if (node < 0 || tok[node] != am[path[j - 1]]) break;
+            if (node < 0) break;
+            if (!MTV_INDEX_OK(node, T, dev_error) || !MTV_INDEX_OK(path[j - 1], T, dev_error)) break;
+            if (tok[node] != am[path[j - 1]]) break;
             len = j;
         }
         atomicMax(&best_key, (unsigned)len * 256u + (255u - (unsigned)p));
@@ -132,10 +134,11 @@ accept_finish_kernel(int T, int K, int P, int ns, const unsigned long long *__re
     const int len = best_key / 256, p = 255 - (int)(best_key % 256);
     if ((int)threadIdx.x <= K) {
         const int j = threadIdx.x;
-        const int node = j <= len ? ri[(size_t)p * (K + 1) + j] : -1;
+        int node = j <= len ? ri[(size_t)p * (K + 1) + j] : -1;
+        if (node >= 0 && !MTV_INDEX_OK(node, T, dev_error)) node = -1;
         acc_nodes[(size_t)b * (K + 1) + j] = node;
         acc_tok[(size_t)b * (K + 1) + j] = node >= 0 ? tok[node] : -1;
-        if (j == len) next_root[b] = am[node];
+        if (j == len && node >= 0) next_root[b] = am[node];
         if (j == 0) { accept_len[b] = len; best_path[b] = p; }
     }
 }
@@ -146,6 +149,7 @@ extern "C" int tree_accept(const mtv_tree_t *tree, int B, int V, const mtv_bf16 
                            int32_t *accept_len, int32_t *best_path, int32_t *acc_nodes, int32_t *acc_tok,
                            int32_t *next_root, void *ws, size_t ws_bytes, void *stream) {
     using namespace mtv;
+    MTV_RANGE("tree_accept");
     if (!tree || !tree->on_device || !logits || !tree_tok || !accept_len || !best_path || !acc_nodes ||
         !acc_tok || !next_root || !ws || B < 1 || V < 1)
         return MTV_ERR_INVALID_ARG;
@@ -162,7 +166,7 @@ extern "C" int tree_accept(const mtv_tree_t *tree, int B, int V, const mtv_bf16 
     }
     TapScope tap(MTV_KERNEL_ACCEPT_FINISH, st);
     accept_finish_kernel<<<B, 128, 0, st>>>(tree->T, tree->K, tree->P, L.nsplit, part, tree_tok, tree->d_retrieve,
-                                            accept_len, best_path, acc_nodes, acc_tok, next_root);
+                                            accept_len, best_path, acc_nodes, acc_tok, next_root, tree->d_error);
     MTV_CUDA_CHECK(cudaGetLastError());
     return MTV_OK;
 }
@@ -173,13 +177,14 @@ extern "C" int tree_accept_keys(const mtv_tree_t *tree, int B, const unsigned lo
                                 int32_t *accept_len, int32_t *best_path, int32_t *acc_nodes, int32_t *acc_tok,
                                 int32_t *next_root, void *stream) {
     using namespace mtv;
+    MTV_RANGE("tree_accept_keys");
     if (!tree || !tree->on_device || !keys || !tree_tok || !accept_len || !best_path || !acc_nodes || !acc_tok ||
         !next_root || B < 1)
         return MTV_ERR_INVALID_ARG;
     if (tree->P > 255) return MTV_ERR_UNSUPPORTED_SHAPE;
     accept_finish_kernel<<<B, 128, 0, (cudaStream_t)stream>>>(tree->T, tree->K, tree->P, 1, keys, tree_tok,
                                                               tree->d_retrieve, accept_len, best_path, acc_nodes,
-                                                              acc_tok, next_root);
+                                                              acc_tok, next_root, tree->d_error);
     MTV_CUDA_CHECK(cudaGetLastError());
     return MTV_OK;
 }
@@ -219,6 +224,7 @@ extern "C" int tree_accept_static_scratch(const mtv_tree_t *tree, int B, int V, 
                                           const int32_t *tree_tok, int32_t *accept_len, int32_t *best_path,
                                           int32_t *acc_nodes, int32_t *acc_tok, int32_t *next_root, void *stream) {
     using namespace mtv;
+    MTV_RANGE("tree_accept_static_scratch");
     if (!tree || !tree->on_device || !logits || !tree_tok || !accept_len || !best_path || !acc_nodes ||
         !acc_tok || !next_root || B < 1 || V < 1)
         return MTV_ERR_INVALID_ARG;
@@ -240,7 +246,7 @@ extern "C" int tree_accept_static_scratch(const mtv_tree_t *tree, int B, int V, 
     node_argmax_partial_kernel<<<dim3(L.nsplit, B * tree->T), ARGMAX_THREADS, 0, st>>>(
         V, reinterpret_cast<const __nv_bfloat16 *>(logits), part);
     accept_finish_kernel<<<B, 128, 0, st>>>(tree->T, tree->K, tree->P, L.nsplit, part, tree_tok, tree->d_retrieve,
-                                            accept_len, best_path, acc_nodes, acc_tok, next_root);
+                                            accept_len, best_path, acc_nodes, acc_tok, next_root, tree->d_error);
     MTV_CUDA_CHECK(cudaGetLastError());
     return MTV_OK;
 }

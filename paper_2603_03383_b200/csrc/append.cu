@@ -8,14 +8,25 @@
 
 namespace mtv {
 
+// One layer (caches given directly) or, with blockIdx.z = layer, all layers of a step in one launch (caches through
+// the device pointer arrays of kv_compact_accepted; q, k_new, v_new then hold the layers back to back).
 __global__ void __launch_bounds__(128)
 tree_kv_append_rope_kernel(int T, int Hq, int Hkv, int D, int Lcap, __nv_bfloat16 *__restrict__ q,
                            const __nv_bfloat16 *__restrict__ k_new, const __nv_bfloat16 *__restrict__ v_new,
-                           __nv_bfloat16 *__restrict__ k_cache, __nv_bfloat16 *__restrict__ v_cache, int64_t sb,
-                           int64_t sh, int64_t st, const int32_t *__restrict__ seq_lens,
+                           __nv_bfloat16 *__restrict__ k_cache, __nv_bfloat16 *__restrict__ v_cache,
+                           __nv_bfloat16 *const *__restrict__ k_caches, __nv_bfloat16 *const *__restrict__ v_caches,
+                           int64_t sb, int64_t sh, int64_t st, const int32_t *__restrict__ seq_lens,
                            const int32_t *__restrict__ depth, double log2_theta, int32_t *__restrict__ status) {
     __shared__ float cs[64], sn[64];   // D / 2 <= 64
     const int i = blockIdx.x, b = blockIdx.y;
+    if (k_caches) {
+        const size_t layer = blockIdx.z, B = gridDim.y;
+        k_cache = k_caches[layer];
+        v_cache = v_caches[layer];
+        q += layer * B * T * Hq * D;
+        k_new += layer * B * T * Hkv * D;
+        v_new += layer * B * T * Hkv * D;
+    }
     const int L = seq_lens[b];
     if (L + T > Lcap) {
         if (status && i == 0 && threadIdx.x == 0) status[b] = MTV_ERR_CAPACITY;
@@ -60,6 +71,7 @@ extern "C" int tree_kv_append_rope(const mtv_tree_t *tree, int B, int Hq, int Hk
                                    int64_t stride_b, int64_t stride_h, int64_t stride_t, int Lcap,
                                    const int32_t *seq_lens, float rope_theta, int32_t *status, void *stream) {
     using namespace mtv;
+    MTV_RANGE("tree_kv_append_rope");
     if (!tree || !tree->on_device || !q || !k_new || !v_new || !k_cache || !v_cache || !seq_lens) return MTV_ERR_INVALID_ARG;
     if (B < 1 || Hq < 1 || Hkv < 1 || Lcap < tree->T || rope_theta < 0.f) return MTV_ERR_INVALID_ARG;
     if ((D != 64 && D != 128) || B > 65535) return MTV_ERR_UNSUPPORTED_SHAPE;
@@ -67,8 +79,30 @@ extern "C" int tree_kv_append_rope(const mtv_tree_t *tree, int B, int Hq, int Hk
     tree_kv_append_rope_kernel<<<dim3(tree->T, B), 128, 0, (cudaStream_t)stream>>>(
         tree->T, Hq, Hkv, D, Lcap, reinterpret_cast<__nv_bfloat16 *>(q), reinterpret_cast<const __nv_bfloat16 *>(k_new),
         reinterpret_cast<const __nv_bfloat16 *>(v_new), reinterpret_cast<__nv_bfloat16 *>(k_cache),
-        reinterpret_cast<__nv_bfloat16 *>(v_cache), stride_b, stride_h, stride_t, seq_lens, tree->d_depth, log2(theta),
-        status);
+        reinterpret_cast<__nv_bfloat16 *>(v_cache), nullptr, nullptr, stride_b, stride_h, stride_t, seq_lens,
+        tree->d_depth, log2(theta), status);
+    MTV_CUDA_CHECK(cudaGetLastError());
+    return MTV_OK;
+}
+
+extern "C" int tree_kv_append_rope_layers(const mtv_tree_t *tree, int B, int Hq, int Hkv, int D, int n_layers,
+                                          mtv_bf16 *q_layers, const mtv_bf16 *k_new_layers, const mtv_bf16 *v_new_layers,
+                                          mtv_bf16 *const *k_caches, mtv_bf16 *const *v_caches, int64_t stride_b,
+                                          int64_t stride_h, int64_t stride_t, int Lcap, const int32_t *seq_lens,
+                                          float rope_theta, int32_t *status, void *stream) {
+    using namespace mtv;
+    MTV_RANGE("tree_kv_append_rope_layers");
+    if (!tree || !tree->on_device || !q_layers || !k_new_layers || !v_new_layers || !k_caches || !v_caches || !seq_lens)
+        return MTV_ERR_INVALID_ARG;
+    if (B < 1 || Hq < 1 || Hkv < 1 || n_layers < 1 || Lcap < tree->T || rope_theta < 0.f) return MTV_ERR_INVALID_ARG;
+    if ((D != 64 && D != 128) || B > 65535 || n_layers > 65535) return MTV_ERR_UNSUPPORTED_SHAPE;
+    const double theta = rope_theta == 0.f ? 10000.0 : (double)rope_theta;
+    tree_kv_append_rope_kernel<<<dim3(tree->T, B, n_layers), 128, 0, (cudaStream_t)stream>>>(
+        tree->T, Hq, Hkv, D, Lcap, reinterpret_cast<__nv_bfloat16 *>(q_layers),
+        reinterpret_cast<const __nv_bfloat16 *>(k_new_layers), reinterpret_cast<const __nv_bfloat16 *>(v_new_layers),
+        nullptr, nullptr, reinterpret_cast<__nv_bfloat16 *const *>(k_caches),
+        reinterpret_cast<__nv_bfloat16 *const *>(v_caches), stride_b, stride_h, stride_t, seq_lens, tree->d_depth,
+        log2(theta), status);
     MTV_CUDA_CHECK(cudaGetLastError());
     return MTV_OK;
 }

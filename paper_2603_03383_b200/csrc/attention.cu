@@ -314,6 +314,7 @@ extern "C" int tree_verify_attention(const mtv_tree_t *tree, int B, int Hq, int 
                                      mtv_bf16 *out, int32_t *status,
                                      void *ws, size_t ws_bytes, void *stream) {
     using namespace mtv;
+    MTV_RANGE("tree_verify_attention");
     if (!tree || !tree->on_device || !q || !k_cache || !v_cache || !seq_lens || !out || !ws) return MTV_ERR_INVALID_ARG;
     if (B < 1 || Hq < 1 || Hkv < 1 || Lcap < tree->T) return MTV_ERR_INVALID_ARG;
     if ((D != 64 && D != 128) || Hq % Hkv != 0 || Hq / Hkv > 8 || B > 65535) return MTV_ERR_UNSUPPORTED_SHAPE;

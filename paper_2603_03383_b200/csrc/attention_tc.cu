@@ -249,7 +249,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     // With more query blocks than CTA pairs fit the device, blocks start in grid order as pairs retire: the longest
     // sequences go first (the order comes from a small kernel in front of this one), so that the last pairs to start
     // are the shortest.
-    const int b = p.order ? p.order[blockIdx.z] : blockIdx.z;
+    int b = p.order ? p.order[blockIdx.z] : blockIdx.z;
+    if (!MTV_INDEX_OK(b, gridDim.z, p.dev_error)) b = blockIdx.z;   // (both CTAs of a pair read the same entry)
     const int L = p.seq_lens[b];
     const int rows0 = blk * 256 + (int)rank * 128;   // first row of this CTA inside the (sequence, KV head) block
     auto tile_of = [&](int j) { return split + j * p.nsplit; };

@@ -87,6 +87,37 @@ struct PerDeviceOnce {
     }
 };
 
+// Index checks of the -DMTV_DEBUG_BOUNDS build: MTV_INDEX_OK(i, n, err) is true when 0 <= i < n; otherwise it
+// records MTV_ERR_BOUNDS in the device error word and is false, and the caller skips the access.  In normal builds
+// it is the constant true and the checks vanish.
+#ifdef MTV_DEBUG_BOUNDS
+__device__ __forceinline__ bool index_ok(long long i, long long n, int32_t *err) {
+    if (i >= 0 && i < n) return true;
+    if (err) atomicExch(err, MTV_ERR_BOUNDS);
+    return false;
+}
+#define MTV_INDEX_OK(i, n, err) ::mtv::index_ok((long long)(i), (long long)(n), (err))
+#else
+#define MTV_INDEX_OK(i, n, err) true
+#endif
+
+// NVTX range around a C-ABI call (visible in a timeline profiler; one indirect call when no tool is attached).
+// -DMTV_NO_NVTX leaves them out.
+#ifndef MTV_NO_NVTX
+}  // namespace mtv
+#include <nvtx3/nvToolsExt.h>
+namespace mtv {
+struct NvtxRange {
+    explicit NvtxRange(const char *name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+    NvtxRange(const NvtxRange &) = delete;
+    NvtxRange &operator=(const NvtxRange &) = delete;
+};
+#define MTV_RANGE(name) ::mtv::NvtxRange mtv_nvtx_range__(name)
+#else
+#define MTV_RANGE(name) do { } while (0)
+#endif
+
 // Optional per-kernel event taps (see mtv_set_kernel_taps).
 struct Tap {
     cudaEvent_t *start = nullptr, *stop = nullptr;

@@ -12,33 +12,37 @@ __global__ void __launch_bounds__(256)
 kv_compact_kernel(int T, int K, int D, int Lcap, __nv_bfloat16 *const *__restrict__ k_caches,
                   __nv_bfloat16 *const *__restrict__ v_caches, int64_t sb, int64_t sh, int64_t st,
                   const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ accept_len,
-                  const int32_t *__restrict__ acc_nodes) {
+                  const int32_t *__restrict__ acc_nodes, int32_t *__restrict__ dev_error) {
     __shared__ uint4 stage[2 * MTV_MAX_K * 16];  // [k|v][j][D/8 <= 16]
     const int g = blockIdx.x, b = blockIdx.y, layer = blockIdx.z;
     const int L = seq_lens[b];
     const int n = accept_len[b];
     if (L + T > Lcap || n <= 0) return;
+    if (!MTV_INDEX_OK(n, K + 1, dev_error)) return;      // accept_len comes from the caller's device memory
     const int vec = D / 8;
     __nv_bfloat16 *kc = k_caches[layer] + b * sb + g * sh;
     __nv_bfloat16 *vc = v_caches[layer] + b * sb + g * sh;
     const int total = 2 * n * vec;
     for (int e = threadIdx.x; e < total; e += blockDim.x) {
         const int which = e / (n * vec), j = (e / vec) % n, c = e % vec;
-        const int src = L + acc_nodes[(size_t)b * (K + 1) + j + 1];
+        const int node = acc_nodes[(size_t)b * (K + 1) + j + 1];
+        const int src = L + node;
         const __nv_bfloat16 *base = which ? vc : kc;
-        stage[e] = *reinterpret_cast<const uint4 *>(base + (int64_t)src * st + c * 8);
+        stage[e] = MTV_INDEX_OK(node, T, dev_error) ? *reinterpret_cast<const uint4 *>(base + (int64_t)src * st + c * 8)
+                                                    : make_uint4(0, 0, 0, 0);
     }
     __syncthreads();
     for (int e = threadIdx.x; e < total; e += blockDim.x) {
         const int which = e / (n * vec), j = (e / vec) % n, c = e % vec;
         __nv_bfloat16 *base = which ? vc : kc;
+        if (!MTV_INDEX_OK(acc_nodes[(size_t)b * (K + 1) + j + 1], T, dev_error)) continue;   // a row that was not read is not written
         *reinterpret_cast<uint4 *>(base + (int64_t)(L + j + 1) * st + c * 8) = stage[e];
     }
 }
 
 // Runs after every compaction block has read seq_lens (next kernel on the stream).
 __global__ void seq_lens_advance_kernel(int B, int T, int Lcap, int32_t *seq_lens, const int32_t *accept_len,
-                                        int32_t *status) {
+                                        int32_t *status, int K, int32_t *dev_error) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
     const int L = seq_lens[b];
@@ -47,6 +51,7 @@ __global__ void seq_lens_advance_kernel(int B, int T, int Lcap, int32_t *seq_len
         return;
     }
     if (status) status[b] = MTV_OK;
+    if (!MTV_INDEX_OK(accept_len[b], K + 1, dev_error)) return;
     seq_lens[b] = L + accept_len[b] + 1;
 }
 
@@ -58,6 +63,7 @@ extern "C" int kv_compact_accepted(const mtv_tree_t *tree, int B, int Hkv, int D
                                    int32_t *seq_lens, const int32_t *accept_len, const int32_t *acc_nodes,
                                    int32_t *status, void *stream) {
     using namespace mtv;
+    MTV_RANGE("kv_compact_accepted");
     if (!tree || !k_caches || !v_caches || !seq_lens || !accept_len || !acc_nodes || B < 1 || Hkv < 1 ||
         n_layers < 1 || Lcap < 1)
         return MTV_ERR_INVALID_ARG;
@@ -70,10 +76,11 @@ extern "C" int kv_compact_accepted(const mtv_tree_t *tree, int B, int Hkv, int D
         kv_compact_kernel<<<dim3(Hkv, B, n_layers), 256, 0, st>>>(
         tree->T, tree->K, D, Lcap, reinterpret_cast<__nv_bfloat16 *const *>(k_caches),
         reinterpret_cast<__nv_bfloat16 *const *>(v_caches), stride_b, stride_h, stride_t, seq_lens, accept_len,
-            acc_nodes);
+            acc_nodes, tree->d_error);
     }
     TapScope tap(MTV_KERNEL_SEQ_ADVANCE, st);
-    seq_lens_advance_kernel<<<(B + 127) / 128, 128, 0, st>>>(B, tree->T, Lcap, seq_lens, accept_len, status);
+    seq_lens_advance_kernel<<<(B + 127) / 128, 128, 0, st>>>(B, tree->T, Lcap, seq_lens, accept_len, status, tree->K,
+                                                                   tree->d_error);
     MTV_CUDA_CHECK(cudaGetLastError());
     return MTV_OK;
 }

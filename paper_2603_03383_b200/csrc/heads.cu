@@ -492,6 +492,7 @@ extern "C" int medusa_heads_topk(const mtv_tree_t *tree, int B, int H, int V,
                                  int32_t *cand, float *cand_logit, int32_t *tree_tok,
                                  void *ws, size_t ws_bytes, void *stream) {
     using namespace mtv;
+    MTV_RANGE("medusa_heads_topk");
     if (!tree || !tree->on_device || !hidden || !W1 || !W2 || !root_tok || !cand || !tree_tok || !ws)
         return MTV_ERR_INVALID_ARG;
     if (B < 1 || H < 8 || V < 1) return MTV_ERR_INVALID_ARG;

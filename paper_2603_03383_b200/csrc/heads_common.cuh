@@ -141,6 +141,7 @@ __device__ __forceinline__ void vocab_tail(const VocabParams &p, const int NB, c
         const int b = b0 + e / p.T, i = e % p.T;
         if (b >= p.B) break;
         const int slot = p.tree_indices[i];
+        if (!MTV_INDEX_OK(slot, p.C, p.dev_error)) continue;
         const int32_t root = p.root_tok[b];
         if (i == 0) p.cand[(size_t)b * p.C] = root;
         p.tree_tok[(size_t)b * p.T + i] = slot == 0 ? root : __ldcg(p.cand + (size_t)b * p.C + slot);

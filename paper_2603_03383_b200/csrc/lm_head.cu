@@ -266,6 +266,7 @@ __global__ void lm_head_finish_kernel(int M, const unsigned long long *__restric
 extern "C" int lm_head_argmax(const mtv_tree_t *tree, int B, int H, int V, const mtv_bf16 *x, const mtv_bf16 *W,
                               int32_t *am, float *am_val, unsigned long long *keys, void *stream) {
     using namespace mtv;
+    MTV_RANGE("lm_head_argmax");
     if (!tree || !tree->on_device || !x || !W || !keys || B < 1 || V < 1 || (am_val && !am)) return MTV_ERR_INVALID_ARG;
     if (H < 64 || H % 64 != 0) return MTV_ERR_UNSUPPORTED_SHAPE;
     if (((uintptr_t)x | (uintptr_t)W) & 15) return MTV_ERR_INVALID_ARG;

@@ -32,11 +32,22 @@ static int step_accept(const mtv_tree_t *tree, const mtv_step_args *a, void *str
                        a->next_root, a->ws, a->ws_bytes, stream);
 }
 
-extern "C" int mtv_verify_step(const mtv_tree_t *tree, const mtv_step_args *a, void *stream) {
-    if (!tree || !a || !a->k_caches_host || !a->v_caches_host) return MTV_ERR_INVALID_ARG;
-    int rc = medusa_heads_topk(tree, a->B, a->H, a->V, a->hidden, a->W1, a->b1, a->W2, a->root_tok, a->cand,
+// One step; root_tok and the optional append are given separately so that a chain of steps can feed a step's root
+// from the previous step's next_root without touching the caller's structs.
+static int verify_step(const mtv_tree_t *tree, const mtv_step_args *a, const int32_t *root_tok,
+                       const mtv_append_args *ap, void *stream) {
+    if (!tree || !a || !a->k_caches_host || !a->v_caches_host || !root_tok) return MTV_ERR_INVALID_ARG;
+    int rc = medusa_heads_topk(tree, a->B, a->H, a->V, a->hidden, a->W1, a->b1, a->W2, root_tok, a->cand,
                                a->cand_logit, a->tree_tok, a->ws, a->ws_bytes, stream);
     if (rc != MTV_OK) return rc;
+    if (ap && (ap->k_new_layers || ap->v_new_layers)) {
+        // the tree nodes' K/V rows of every layer, in one launch in front of the first attention (which starts its
+        // set-up under this kernel's tail: programmatic dependent launch)
+        rc = tree_kv_append_rope_layers(tree, a->B, a->Hq, a->Hkv, a->D, a->n_layers, const_cast<mtv_bf16 *>(a->q_layers),
+                                        ap->k_new_layers, ap->v_new_layers, a->k_caches, a->v_caches, a->stride_b,
+                                        a->stride_h, a->stride_t, a->Lcap, a->seq_lens, ap->rope_theta, a->status, stream);
+        if (rc != MTV_OK) return rc;
+    }
     const size_t per_layer = (size_t)a->B * tree->T * a->Hq * a->D;
     for (int l = 0; l < a->n_layers; ++l) {
         rc = tree_verify_attention(tree, a->B, a->Hq, a->Hkv, a->D, a->q_layers + l * per_layer, a->k_caches_host[l],
@@ -49,6 +60,32 @@ extern "C" int mtv_verify_step(const mtv_tree_t *tree, const mtv_step_args *a, v
     return kv_compact_accepted(tree, a->B, a->Hkv, a->D, a->n_layers, a->k_caches, a->v_caches, a->stride_b,
                                a->stride_h, a->stride_t, a->Lcap, a->seq_lens, a->accept_len, a->acc_nodes, a->status,
                                stream);
+}
+
+extern "C" int mtv_verify_step(const mtv_tree_t *tree, const mtv_step_args *a, void *stream) {
+    MTV_RANGE("mtv_verify_step");
+    if (!a) return MTV_ERR_INVALID_ARG;
+    return verify_step(tree, a, a->root_tok, nullptr, stream);
+}
+
+// n steps back to back on one stream.  Nothing is decided on the host between them: step s + 1 takes its root token
+// from step s's next_root and its prefix lengths from the seq_lens that step s's compaction advanced, both on the device.
+extern "C" int mtv_verify_steps(const mtv_tree_t *tree, const mtv_step_args *steps, const mtv_append_args *appends,
+                                int n_steps, void *stream) {
+    MTV_RANGE("mtv_verify_steps");
+    if (!tree || !steps || n_steps < 1) return MTV_ERR_INVALID_ARG;
+    for (int s = 0; s < n_steps; ++s) {      // the whole chain is looked at before anything is enqueued
+        if (!steps[s].root_tok && (s == 0 || !steps[s - 1].next_root)) return MTV_ERR_INVALID_ARG;
+        if (!steps[s].seq_lens || steps[s].seq_lens != steps[0].seq_lens) return MTV_ERR_INVALID_ARG;   // one chain, one set of lengths
+        if (!steps[s].k_caches_host || !steps[s].v_caches_host) return MTV_ERR_INVALID_ARG;
+    }
+    for (int s = 0; s < n_steps; ++s) {
+        const mtv_step_args *a = steps + s;
+        const int32_t *root = a->root_tok ? a->root_tok : steps[s - 1].next_root;
+        const int rc = verify_step(tree, a, root, appends ? appends + s : nullptr, stream);
+        if (rc != MTV_OK) return rc;
+    }
+    return MTV_OK;
 }
 
 namespace {
@@ -85,6 +122,7 @@ int host_step_aux(HostStepAux **out) {
 // down on a second copy stream in up to sixteen groups of layers while later layers are still running.
 extern "C" int mtv_verify_step_host(const mtv_tree_t *tree, const mtv_step_args *d, const mtv_step_args *h,
                                     void *stream) {
+    MTV_RANGE("mtv_verify_step_host");
     if (!tree || !d || !h || !d->k_caches_host || !d->v_caches_host) return MTV_ERR_INVALID_ARG;
     HostStepAux *aux = nullptr;
     if (host_step_aux(&aux) != MTV_OK) return MTV_ERR_CUDA;
@@ -164,6 +202,14 @@ __global__ void selftest_wait_timeout_kernel(int32_t *dev_error) {
     if (!ok && threadIdx.x == 0) atomicExch(dev_error, MTV_ERR_TIMEOUT);
 }
 }  // namespace
+
+extern "C" int mtv_debug_bounds_enabled(void) {
+#ifdef MTV_DEBUG_BOUNDS
+    return 1;
+#else
+    return 0;
+#endif
+}
 
 extern "C" int mtv_selftest_wait_timeout(const mtv_tree_t *tree, void *stream) {
     if (!tree || !tree->on_device) return MTV_ERR_INVALID_ARG;

@@ -108,7 +108,7 @@ TID_Q, TID_K, TID_V = 100, 200, 300  # + layer
 
 @dataclasses.dataclass(frozen=True)
 class Workload:
-    """Shapes of one benchmark configuration (notation of the scope table)."""
+    """Shapes of one benchmark configuration (H hidden size, V vocabulary, K heads, T tree nodes, L prefix length, Hq/Hkv query and KV heads, D head size)."""
     name: str
     cfg_id: int
     B: int

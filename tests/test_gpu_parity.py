@@ -584,3 +584,128 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
     assert binding.mtv_device_error(tree) == 0
     _attention_case(tb, tree, 1, 8, 2, 128, [300], seed=3)
     assert binding.mtv_device_error(tree) == 0
+
+
+@pytest.mark.parametrize("lm_head", [False, True])
+def test_verify_steps_chain_in_one_call(lm_head):
+    """Three steps through mtv_verify_steps, enqueued by ONE call with every step's inputs laid out beforehand: each
+    step appends its tree's K/V rows (all layers in one launch, rotary embedding at seq_lens + depth), attends,
+    accepts and compacts; the next step's root token and prefix lengths reach it on the device only.  Every
+    step's outputs and the final caches equal the checker stepping the same way."""
+    B, H, V, Hq, Hkv, D, K, n_layers, n_steps = 2, 256, 2000, 8, 2, 128, 4, 3, 3
+    tb, tree = make_tree("rank_prior", K, (), 64)
+    T = tree.T
+    lens0 = [131, 20]
+    Lcap = max(lens0) + n_steps * (K + 1) + T
+    seed = 177
+    kc = [synth.normal_bf16(seed, 500 + l, (B, Hkv, Lcap, D)) for l in range(n_layers)]
+    vc = [synth.normal_bf16(seed, 600 + l, (B, Hkv, Lcap, D)) for l in range(n_layers)]
+    kd, vd = [t.to(DEV) for t in kc], [t.to(DEV) for t in vc]
+    sl_ref = torch.tensor(lens0, dtype=torch.int32)
+    sl_dev = sl_ref.to(DEV)
+    root_ref = synth.uniform_int(seed, 7, B, 0, V - 1).to(torch.int32)
+    root0_dev = root_ref.to(DEV)
+    ws = workspace(tree, B, H, V, Hq, Hkv, D, Lcap)
+    kp, vp = binding.cache_pointer_array(kd, DEV), binding.cache_pointer_array(vd, DEV)
+    kph, vph = binding.cache_pointer_array(kd), binding.cache_pointer_array(vd)
+    W_lm = synth.normal_bf16(seed, 901, (V, H))
+    W_lm_dev = W_lm.to(DEV)
+    steps, appends, keep, want = [], [], [], []
+    for s in range(n_steps):
+        # ---- the checker's step s, which also fixes the inputs of step s
+        s_in = seed + 10 * s
+        for attempt in range(20):
+            hidden, W1, b1, W2, _ = synth.head_inputs(B, H, V, K, s_in)
+            z = ref.heads_logits(hidden, W1, b1, W2)
+            cand_ref, _, tt_ref, gap = ref.heads_candidates(z, root_ref, tb)
+            if gap > 1e-5 * z.abs().max().item():
+                break
+            s_in += 1000
+        q = torch.stack([synth.normal_bf16(s_in, 700 + l, (B, T, Hq, D)) for l in range(n_layers)])
+        kn = torch.stack([synth.normal_bf16(s_in, 800 + l, (B, T, Hkv, D)) for l in range(n_layers)])
+        vn = torch.stack([synth.normal_bf16(s_in, 900 + l, (B, T, Hkv, D)) for l in range(n_layers)])
+        logits, planted = synth.planted_logits(B, T, V, K, tt_ref, tb["parent"], tb["rank"], s_in, p_accept=(0.9, 0.6))
+        am_ref = ref.node_argmax(logits)
+        out_ref = []
+        for l in range(n_layers):
+            q_rot, k_rot = ref.rope(q[l], kn[l], sl_ref.tolist(), tb["depth"])
+            for b in range(B):
+                L = int(sl_ref[b])
+                kc[l][b, :, L:L + T] = k_rot[b].to(torch.bfloat16).permute(1, 0, 2)
+                vc[l][b, :, L:L + T] = vn[l][b].permute(1, 0, 2)
+            out_ref.append(ref.tree_attention(q_rot.to(torch.bfloat16), kc[l], vc[l], sl_ref, tb["mask"]))
+        acc_ref = ref.tree_accept(am_ref, tt_ref, tb)
+        assert torch.equal(acc_ref["accept_len"], planted)
+        for l in range(n_layers):
+            kc[l], new_len = ref.kv_compact(kc[l], sl_ref, acc_ref["accept_len"], acc_ref["acc_nodes"])
+            vc[l], _ = ref.kv_compact(vc[l], sl_ref, acc_ref["accept_len"], acc_ref["acc_nodes"])
+        want.append(dict(tree_tok=tt_ref, cand=cand_ref, out=out_ref, acc=acc_ref, seq_lens=new_len))
+        # ---- this library's step s: buffers and the struct, nothing launched yet
+        dev = dict(hidden=hidden.to(DEV), W1=W1.to(DEV), b1=b1.to(DEV), W2=W2.to(DEV), q_layers=q.to(DEV),
+                   seq_lens=sl_dev, cand=_i32(B, tree.C), tree_tok=_i32(B, T),
+                   out_layers=torch.zeros(n_layers, B, T, Hq, D, dtype=torch.bfloat16, device=DEV),
+                   accept_len=_i32(B), best_path=_i32(B), acc_nodes=_i32(B, K + 1), acc_tok=_i32(B, K + 1),
+                   next_root=_i32(B), status=_i32(B), k_caches=kp, v_caches=vp, k_caches_host=kph, v_caches_host=vph, ws=ws)
+        if lm_head:     # the same next tokens as the argmax of an LM head over hidden states built around its rows
+            x_final = (W_lm[am_ref.flatten().long()].float().reshape(B, T, H) +
+                       0.3 * synth.normal_bf16(s_in, 902, (B, T, H)).float()).to(torch.bfloat16)
+            am, zmax, z2 = ref.lm_head_argmax(x_final.reshape(B * T, H), W_lm)
+            assert torch.equal(am.long(), am_ref.flatten().long()) and ((zmax - z2) > 1e-3 * zmax.abs().max()).all()
+            dev["x_final"], dev["W_lm"] = x_final.to(DEV), W_lm_dev
+        else:
+            dev["logits"] = logits.to(DEV)
+        if s == 0:
+            dev["root_tok"] = root0_dev      # later steps: NULL = the previous step's next_root, on the device
+        a = binding.StepArgs()
+        a.B, a.H, a.V, a.Hq, a.Hkv, a.D, a.n_layers, a.Lcap = B, H, V, Hq, Hkv, D, n_layers, Lcap
+        a.stride_b, a.stride_h, a.stride_t, a.scale = Hkv * Lcap * D, Lcap * D, D, 0.0
+        for name, t in dev.items():
+            setattr(a, name, t.data_ptr())
+        a.ws_bytes = ws.numel()
+        ap = binding.AppendArgs()
+        kn_d, vn_d = kn.to(DEV), vn.to(DEV)
+        ap.k_new_layers, ap.v_new_layers, ap.rope_theta = kn_d.data_ptr(), vn_d.data_ptr(), 0.0
+        steps.append(a)
+        appends.append(ap)
+        keep.append((dev, kn_d, vn_d))
+        sl_ref, root_ref = new_len, acc_ref["next_root"]
+    # ---- one call, then everything is compared
+    torch.cuda.synchronize()
+    binding.mtv_verify_steps(tree, steps, appends)
+    torch.cuda.synchronize()
+    assert binding.mtv_device_error(tree) == 0
+    for s in range(n_steps):
+        dev, w = keep[s][0], want[s]
+        assert dev["status"].tolist() == [0] * B
+        assert torch.equal(dev["tree_tok"].cpu(), w["tree_tok"]) and torch.equal(dev["cand"].cpu(), w["cand"]), s
+        for l in range(n_layers):
+            assert_close(dev["out_layers"][l], w["out"][l], "step %d layer %d" % (s, l))
+        for name in ("accept_len", "best_path", "acc_nodes", "acc_tok", "next_root"):
+            assert torch.equal(dev[name].cpu(), w["acc"][name]), (s, name)
+    assert torch.equal(sl_dev.cpu(), sl_ref) and int(sl_ref.min()) > min(lens0)
+    for l in range(n_layers):
+        for b in range(B):
+            n, n0 = int(sl_ref[b]), lens0[b]
+            assert torch.equal(vd[l][b, :, :n].cpu(), vc[l][b, :, :n])
+            assert torch.equal(kd[l][b, :, :n0].cpu(), kc[l][b, :, :n0])
+            assert_close(kd[l][b, :, :n], kc[l][b, :, :n], "compacted K rows")
+
+
+def test_verify_steps_refuses_a_chain_without_a_first_root_or_with_two_length_arrays():
+    tb, tree = make_tree("cartesian", 3, (4, 2, 2))
+    a, b = binding.StepArgs(), binding.StepArgs()
+    two = torch.zeros(2, 4, dtype=torch.int32, device=DEV)
+    ptrs = torch.zeros(1, dtype=torch.int64)
+    for x in (a, b):
+        x.k_caches_host = x.v_caches_host = ptrs.data_ptr()
+        x.seq_lens = two[0].data_ptr()
+    with pytest.raises(binding.MtvError) as e:
+        binding.mtv_verify_steps(tree, [a])                       # root_tok NULL in the first step
+    assert e.value.code == -1
+    a.root_tok = a.next_root = two[1].data_ptr()
+    b.seq_lens = two[1].data_ptr()                                # the second step names other lengths
+    with pytest.raises(binding.MtvError) as e:
+        binding.mtv_verify_steps(tree, [a, b])                    # refused before the first step is enqueued
+    assert e.value.code == -1
+    torch.cuda.synchronize()
+    assert binding.mtv_device_error(tree) == 0
