@@ -43,6 +43,10 @@ def parse():
     ap.add_argument("--repeats", type=int, default=5, help="timed repeats of --steps; the median is reported")
     ap.add_argument("--no-other-workloads", action="store_true", help="skip the short runs of the other four configurations")
     ap.add_argument("--no-parity-gate", action="store_true", help="skip the checks against the CPU checker before timing")
+    ap.add_argument("--shard", default="sequence", choices=["sequence", "kvhead"],
+                    help="how N GPUs share the work: 'sequence' = every rank verifies its own sequences (no collective, "
+                         "weak scaling); 'kvhead' = all ranks work on the SAME sequences, heads split by vocabulary slab "
+                         "and attention by KV head with an all-gather after each (strong scaling)")
     ap.add_argument("--overhead-sweep", action="store_true",
                     help="instead of the step benchmark: time tree attention (T nodes) against single-token decode "
                          "attention (a root-only tree) over prefix lengths, the attention part of the paper's overhead ratio")
@@ -476,6 +480,167 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_sharded(args):
+    """--shard kvhead: all ranks verify the same sequences.  Rank r projects the heads onto its vocabulary slab and
+    attends with its KV heads; one all-gather after each brings the pieces into local memory, where the library's
+    merge kernels put them together; acceptance runs on every rank (the logits are replicated), compaction on the
+    rank's own caches.  Total work is fixed as N grows: "scaling": "strong"."""
+    import torch
+    import torch.distributed as dist
+    from paper_2603_03383_b200 import binding, sharded, synth
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    w = synth.WORKLOADS[args.workload]
+    n_layers = args.layers
+    P = build_problem(w, n_layers, dev, seed=w.seed)             # the same sequences on every rank
+    tree, B, T = P["tree"], w.B, P["tree"].T
+    K_steps, W_steps = args.steps, max(args.warmup, 3)
+    gate = None
+    if rank == 0 and not args.no_parity_gate:
+        try:
+            gate = parity_gate(w, P, n_layers)                    # the unsplit path against the CPU checker
+        except ParityError as e:
+            print(json.dumps({"metric": METRIC, "value": None, "unit": UNIT, "error": "parity gate failed: %s" % e,
+                              "config": {"workload": workload_string(w, T, n_layers)}}))
+            sys.exit(1)
+    else:
+        P["seq_lens"].copy_(P["seq_lens0"])
+        binding.mtv_verify_step(tree, P["args"])
+    torch.cuda.synchronize()
+    whole = {n: P[n].clone() for n in ("cand", "tree_tok", "accept_len", "best_path", "acc_nodes", "acc_tok", "next_root",
+                                       "seq_lens")}
+    # the unsplit attention of the last layer on the caches as that step's compaction left them (the state the slices
+    # below are cut from)
+    whole_out = torch.zeros_like(P["out_layers"][n_layers - 1])
+    binding.tree_verify_attention(tree, P["q_layers"][n_layers - 1], P["k_list"][n_layers - 1], P["v_list"][n_layers - 1],
+                                  P["seq_lens0"], whole_out, P["ws"])
+    torch.cuda.synchronize()
+    # ---- this rank's slices (a rank of a real job would load only these)
+    pl = sharded.plan(rank, world, w.V, w.Hq, w.Hkv, max_kd=max(tree.k_d))
+    W2_slab = P["W2"][:, pl.v_lo:pl.v_hi].contiguous()
+    q_l = P["q_layers"][:, :, :, pl.q_lo:pl.q_lo + pl.hq_local].contiguous()
+    k_l = [k[:, pl.kv_lo:pl.kv_lo + pl.hkv_local].contiguous() for k in P["k_list"]]
+    v_l = [v[:, pl.kv_lo:pl.kv_lo + pl.hkv_local].contiguous() for v in P["v_list"]]
+    if world > 1:
+        del P["W2"], P["k_list"], P["v_list"]
+        torch.cuda.empty_cache()
+    kp, vp = binding.cache_pointer_array(k_l, dev), binding.cache_pointer_array(v_l, dev)
+    Lcap = P["Lcap"]
+    strides = (pl.hkv_local * Lcap * w.D, Lcap * w.D, w.D)
+    out_layers = torch.zeros(n_layers, B, T, w.Hq, w.D, dtype=torch.bfloat16, device=dev)
+
+    def step():
+        P["seq_lens"].copy_(P["seq_lens0"])
+        sharded.medusa_heads_topk_sharded(tree, pl, P["hidden"], P["W1"], P["b1"], W2_slab, P["root_tok"], P["cand"],
+                                          P["cand_logit"], P["tree_tok"], P["ws"])
+        for l in range(n_layers):
+            sharded.tree_verify_attention_sharded(tree, pl, q_l[l], k_l[l], v_l[l], P["seq_lens"], out_layers[l], P["ws"],
+                                                  status=P["status"])
+        binding.tree_accept(tree, P["logits"], P["tree_tok"], P["accept_len"], P["best_path"], P["acc_nodes"],
+                            P["acc_tok"], P["next_root"], P["ws"])
+        binding.kv_compact_accepted(tree, kp, vp, n_layers, B, pl.hkv_local, w.D, strides, Lcap, P["seq_lens"],
+                                    P["accept_len"], P["acc_nodes"], status=P["status"])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # the split step must give what the unsplit one gave (integers bit-exact; attention within the float tolerance:
+    # the key splits of a call depend on how many heads it serves)
+    step()
+    barrier()
+    for n, t in whole.items():
+        if not torch.equal(P[n], t):
+            print(json.dumps({"metric": METRIC, "value": None, "unit": UNIT,
+                              "error": "split step: %s differs from the unsplit step on rank %d" % (n, rank)}))
+            sys.exit(1)
+    err = (out_layers[n_layers - 1].float() - whole_out.float()).abs().max().item()
+    tol = 1e-2 * whole_out.float().abs().max().item() + 1e-3
+    if not err <= tol:
+        print(json.dumps({"metric": METRIC, "value": None, "unit": UNIT,
+                          "error": "split step: attention differs from the unsplit step by %.3e on rank %d" % (err, rank)}))
+        sys.exit(1)
+    for _ in range(W_steps):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    runs_ms = []
+    for _ in range(max(1, args.repeats)):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(K_steps):
+            step()
+        e1.record()
+        barrier()
+        runs_ms.append(max_over_ranks(e0.elapsed_time(e1), world, dev))
+    clocks = sampler.stop() if rank == 0 else None
+    ms_step = statistics.median(runs_ms) / K_steps
+    # end to end: the step's inputs from pinned host memory, its results back to the host, every step
+    host = {n: P[n].cpu().pin_memory() for n in ("hidden", "root_tok", "logits")}
+    host["q"] = q_l.cpu().pin_memory()
+    back = {n: torch.empty_like(P[n], device="cpu").pin_memory() for n in ("tree_tok", "accept_len", "best_path",
+                                                                          "acc_nodes", "acc_tok", "next_root", "seq_lens")}
+    back["out"] = torch.empty_like(out_layers, device="cpu").pin_memory()
+
+    def e2e_step():
+        for n in ("hidden", "root_tok", "logits"):
+            P[n].copy_(host[n], non_blocking=True)
+        q_l.copy_(host["q"], non_blocking=True)
+        step()
+        for n in back:
+            back[n].copy_(out_layers if n == "out" else P[n], non_blocking=True)
+        torch.cuda.synchronize()
+
+    e2e_steps = max(3, min(K_steps, 20))
+    e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_s = max_over_ranks((time.perf_counter() - t0) / e2e_steps, world, dev)
+    h2d = sum(t.numel() * t.element_size() for t in host.values())
+    d2h = sum(t.numel() * t.element_size() for t in back.values())
+    if rank == 0:
+        pk = peaks()
+        alg = algorithmic_bytes(w, tree, n_layers, P["lens"].tolist())
+        gathered = 2 * B * (tree.C * 4 + (tree.C - 1) * 4) + n_layers * B * T * w.Hq * w.D * 2
+        out = {
+            "metric": METRIC, "value": 1000.0 / ms_step, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W_steps,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": workload_string(w, T, n_layers),
+                       "parallelism": "one sequence set on %d GPU(s): heads by vocabulary slab (%d rows each), attention "
+                                      "by KV head (%d of %d each), all-gather + merge kernel after each" % (
+                                          world, pl.v_slab, pl.hkv_local, w.Hkv),
+                       "timing": "median of %d runs of %d steps (%s ms each), stream launches" % (
+                           len(runs_ms), K_steps, ", ".join("%.1f" % r for r in runs_ms)),
+                       "l2": "inputs larger than L2: %.2f GB streamed per step over all ranks" % (alg["step"] / 1e9),
+                       "collective_bytes_per_step_per_rank": gathered, "seed": w.seed, "context": PAPER_CONTEXT},
+            "clocks": clocks,
+            "e2e": {"value": 1.0 / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps},
+            "gpu_launches": K_steps * (LAUNCHES_PER_STEP(n_layers) + 2 + n_layers),
+            "device_error": binding.mtv_device_error(tree, clear=False),
+            "parity_gate": dict(gate or {}, split="integers bit-exact, attention max |diff| %.2e <= %.2e against the unsplit "
+                                "step" % (err, tol)) if gate is not None else "skipped",
+            "step_roofline": {"algorithmic_bytes": alg["step"], "achieved_gbs": alg["step"] / ms_step / 1e6,
+                              "frac_of_measured": alg["step"] / ms_step / 1e6 / (pk["hbm_gbs"] * world)},
+        }
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def quick_workload(name, n_layers, dev, pk, steps=5, repeats=3):
     """A short measurement of one of the other configurations: whole steps (graph replay and plain stream launches:
     their difference is the launch overhead), the attention call alone, and the roofline fractions that go with them.
@@ -776,5 +941,7 @@ if __name__ == "__main__":
         sys.exit(0)
     if a.impl == "reference":
         run_reference(a)
+    elif a.shard == "kvhead":
+        run_sharded(a)
     else:
         run_ours(a)

@@ -362,6 +362,32 @@ int mtv_verify_step_host(const mtv_tree_t *tree, const mtv_step_args *dev, const
                          void *stream);
 
 /* ---------------------------------------------------------------------------
+ * One sequence's step split over several GPUs (the paper runs on one device and has no counterpart; the
+ * split follows its structure: the heads of Section 3.1 are independent over the vocabulary, the tree
+ * attention of Section 3.2 over KV heads).  Each rank runs the ordinary calls on its slice — medusa_heads_topk
+ * on the vocabulary slab [r * v_slab, min(V, (r+1) * v_slab)) of W2 (W1 replicated), tree_verify_attention on
+ * its Hkv / n KV heads and their Hq / n query heads, lm_head_argmax on its slab of W_lm —, a collective outside
+ * this library (NCCL all-gather) brings all ranks' results into LOCAL buffers, and the calls below merge them.
+ * No kernel of this library is ever given another GPU's memory.  All pointers device.
+ *
+ * heads_merge_shards: cand_shards [n_shards][B][C] (ids local to the slab, slot 0 unused), logit_shards
+ *   [n_shards][B][C-1] as medusa_heads_topk wrote them on each rank -> cand, cand_logit (may be NULL), tree_tok
+ *   as medusa_heads_topk on the whole vocabulary writes them: per head the k_d best of the n_shards * k_d entries
+ *   by (logit descending, global id ascending), the same order, so the ids are identical.  Every slab must hold
+ *   at least max k_d rows.  ws: B * 4 bytes.  n_shards <= 16.
+ * attn_interleave_shards: gathered [n_shards][rows][Hq_local][D] (rows = B * T) -> out [rows][n_shards * Hq_local][D].
+ * keys_merge_shards: key_shards [n_shards][n] from lm_head_argmax on each slab (n = B * T) -> keys [n] for
+ *   tree_accept_keys, the slab offsets folded into the index half; ties across slabs go to the lowest global id.
+ */
+int heads_merge_shards(const mtv_tree_t *tree, int B, int n_shards, int v_slab, const int32_t *cand_shards,
+                       const float *logit_shards, const int32_t *root_tok, int32_t *cand, float *cand_logit,
+                       int32_t *tree_tok, void *ws, size_t ws_bytes, void *stream);
+int attn_interleave_shards(int rows, int n_shards, int Hq_local, int D, const mtv_bf16 *gathered, mtv_bf16 *out,
+                           void *stream);
+int keys_merge_shards(int n, int n_shards, int v_slab, const unsigned long long *key_shards,
+                      unsigned long long *keys, void *stream);
+
+/* ---------------------------------------------------------------------------
  * Measurement aid (the paper has no counterpart): per-kernel device timing.
  * While taps are set for a kernel id, every launch of that kernel by this library is
  * bracketed by cudaEventRecord(start[i]) / cudaEventRecord(stop[i]) on the launch

@@ -31,7 +31,8 @@ EXPORTS = ["tree_build_static", "tree_gen_cartesian", "tree_gen_rank_prior", "tr
            "mtv_set_kernel_taps", "mtv_kernel_taps_used", "mtv_device_error",
            "tree_accept_static_scratch", "tree_accept_static_scratch_capacity", "tree_kv_append_rope",
            "lm_head_argmax", "tree_accept_keys", "mtv_selftest_wait_timeout", "tree_kv_append_rope_layers",
-           "mtv_verify_steps", "mtv_debug_bounds_enabled"]
+           "mtv_verify_steps", "mtv_debug_bounds_enabled", "heads_merge_shards", "attn_interleave_shards",
+           "keys_merge_shards"]
 
 
 class MtvError(RuntimeError):
@@ -115,6 +116,9 @@ def lib():
         L.mtv_selftest_wait_timeout.argtypes = [vp, vp]
         L.tree_kv_append_rope_layers.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, i64, i64, i64, i32, vp,
                                                  C.c_float, vp, vp]
+        L.heads_merge_shards.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.attn_interleave_shards.argtypes = [i32, i32, i32, i32, vp, vp, vp]
+        L.keys_merge_shards.argtypes = [i32, i32, i32, vp, vp, vp]
         L.mtv_verify_steps.argtypes = [vp, C.POINTER(StepArgs), C.POINTER(AppendArgs), i32, vp]
         _lib = L
     return _lib
@@ -314,6 +318,28 @@ def kv_compact_accepted(tree, k_ptrs, v_ptrs, n_layers, B, Hkv, D, strides, Lcap
 
 def mtv_verify_step(tree, args: StepArgs, stream=None):
     _check(lib().mtv_verify_step(tree.handle, C.byref(args), _stream(stream)), "mtv_verify_step")
+
+
+def heads_merge_shards(tree, v_slab, cand_shards, logit_shards, root_tok, cand, cand_logit, tree_tok, ws, stream=None):
+    """cand_shards [n][B][C], logit_shards [n][B][C-1] (every rank's medusa_heads_topk results, gathered)."""
+    n, B, _ = cand_shards.shape
+    p, nbytes = _ws(ws)
+    _check(lib().heads_merge_shards(tree.handle, B, n, v_slab, _ptr(cand_shards), _ptr(logit_shards), _ptr(root_tok),
+                                    _ptr(cand), _ptr(cand_logit), _ptr(tree_tok), p, nbytes, _stream(stream)),
+           "heads_merge_shards")
+
+
+def attn_interleave_shards(gathered, out, stream=None):
+    """gathered [n][B][T][Hq_local][D] -> out [B][T][n * Hq_local][D]."""
+    n, B, T, Hl, D = gathered.shape
+    _check(lib().attn_interleave_shards(B * T, n, Hl, D, _ptr(gathered), _ptr(out), _stream(stream)),
+           "attn_interleave_shards")
+
+
+def keys_merge_shards(v_slab, key_shards, keys, stream=None):
+    """key_shards [n][B*T] (int64 storage of the uint64 keys) -> keys [B*T]."""
+    n, m = key_shards.shape
+    _check(lib().keys_merge_shards(m, n, v_slab, _ptr(key_shards), _ptr(keys), _stream(stream)), "keys_merge_shards")
 
 
 def mtv_verify_steps(tree, steps: Sequence[StepArgs], appends: Optional[Sequence[AppendArgs]] = None, stream=None):
