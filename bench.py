@@ -896,7 +896,7 @@ def run_reference(args):
 def run_overhead_sweep(args):
     """Attention part of the paper's Overhead = Time_speculative / Time_autoregressive (Eq. 3) on this GPU:
     the T-node tree attention call against the same call with a root-only tree (one query token), per
-    prefix length, on 32 rotating KV caches.  One JSON line per length."""
+    prefix length, on 32 rotating KV caches (median of five runs of 5 x 32 calls).  One JSON line per length."""
     import torch
     from paper_2603_03383_b200 import binding, synth
     torch.cuda.set_device(0)
@@ -920,14 +920,17 @@ def run_overhead_sweep(args):
             for l in range(layers):
                 binding.tree_verify_attention(tree, qs[l], ks[l], vs[l], sl, out, ws)
             torch.cuda.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            for _ in range(reps):
-                for l in range(layers):
-                    binding.tree_verify_attention(tree, qs[l], ks[l], vs[l], sl, out, ws)
-            e1.record()
-            torch.cuda.synchronize()
-            res[name] = e0.elapsed_time(e1) * 1e3 / (reps * layers)
+            runs = []
+            for _ in range(5):      # the median of five timed runs: single runs of a call this short scatter by a microsecond
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(reps):
+                    for l in range(layers):
+                        binding.tree_verify_attention(tree, qs[l], ks[l], vs[l], sl, out, ws)
+                e1.record()
+                torch.cuda.synchronize()
+                runs.append(e0.elapsed_time(e1) * 1e3 / (reps * layers))
+            res[name] = statistics.median(runs)
             del qs, ks, vs
         print(json.dumps({"prefix": L, "tree_nodes": trees["tree"].T, "us_tree_attention": res["tree"],
                           "us_single_token_attention": res["single"],
