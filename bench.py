@@ -403,6 +403,7 @@ def run_ours(args):
     alg = algorithmic_bytes(w, tree, n_layers, P["lens"].tolist())
     lm = time_lm_head(tree, w, P, dev)
     lm_step_ms = time_step_with_lm_head(tree, w, P, dev, args.launch, max(3, min(K_steps, 20)))
+    chain_ms = time_chained_steps(tree, w, P, dev, args.launch, max(3, min(K_steps, 10)))
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W_steps,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -463,7 +464,12 @@ def run_ours(args):
             "what": "the same step with the acceptance fed by the fused LM head (x_final, W_lm) instead of stored logits",
             "ms_per_step": lm_step_ms, "steps_per_s": 1000.0 / lm_step_ms,
             "algorithmic_bytes": alg["step"] - alg["accept"] + lm_bytes,
-            "frac_of_measured_hbm": (alg["step"] - alg["accept"] + lm_bytes) / lm_step_ms / 1e6 / pk["hbm_gbs"]}}
+            "frac_of_measured_hbm": (alg["step"] - alg["accept"] + lm_bytes) / lm_step_ms / 1e6 / pk["hbm_gbs"]},
+        "chained_steps_with_append": {
+            "what": "mtv_verify_steps: chains of two steps per call, each step first appending its tree's K/V rows with the "
+                    "rotary embedding (all layers, one launch); root token and prefix lengths pass between the steps on the device; "
+                    "the chain starts K + 1 rows short of the configured prefix so that both links fit the caches",
+            "ms_per_step": chain_ms, "steps_per_s": 1000.0 / chain_ms}}
     if not args.no_cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(w, P, n_layers, budget_s=20.0)
     if not args.no_other_workloads and world == 1:
@@ -770,6 +776,58 @@ def time_step_with_lm_head(tree, w, P, dev, launch, steps):
     e1.record()
     torch.cuda.synchronize()
     return e0.elapsed_time(e1) / steps
+
+
+def time_chained_steps(tree, w, P, dev, launch, steps, n_chain=2):
+    """ms per step of mtv_verify_steps: chains of `n_chain` steps in one call, each step first appending its tree's
+    K/V rows (rotary embedding, all layers in one launch), the next step's root token and prefix lengths passed on the
+    device.  Same per-step inputs for every link of the chain (the timing does not depend on the values)."""
+    import torch
+    from paper_2603_03383_b200 import binding, synth
+    n_layers = P["q_layers"].shape[0]
+    kn = synth.normal_bf16(w.seed, 78, (n_layers, w.B, tree.T, w.Hkv, w.D), device=dev)
+    vn = synth.normal_bf16(w.seed, 79, (n_layers, w.B, tree.T, w.Hkv, w.D), device=dev)
+    chain, appends = [], []
+    for s in range(n_chain):
+        a = binding.StepArgs.from_buffer_copy(P["args"])
+        if s > 0:
+            a.root_tok = None                       # = the previous step's next_root
+        ap = binding.AppendArgs()
+        ap.k_new_layers, ap.v_new_layers, ap.rope_theta = kn.data_ptr(), vn.data_ptr(), 0.0
+        chain.append(a)
+        appends.append(ap)
+
+    # every link must fit the caches' capacity (prefix + tree rows): the chain starts (n_chain - 1) (K + 1) rows short of
+    # the configured prefix
+    start = (P["seq_lens0"] - (n_chain - 1) * (w.K + 1)).clamp_(min=0)
+
+    def run_chain():
+        P["seq_lens"].copy_(start)
+        binding.mtv_verify_steps(tree, chain, appends)
+    for _ in range(2):
+        run_chain()
+    torch.cuda.synchronize()
+    if any(P["status"].cpu().tolist()) or int((P["seq_lens"] - start).min()) < n_chain:
+        raise RuntimeError("chained steps: a link was refused (status %s)" % P["status"].cpu().tolist())
+    run = run_chain
+    if launch == "graph":
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                run_chain()
+        torch.cuda.current_stream().wait_stream(side)
+        run = graph.replay
+        run()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / (steps * n_chain)
 
 
 def _sample_plan(w, T, n_layers, est_full_s, budget_s):

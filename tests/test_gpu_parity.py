@@ -709,3 +709,80 @@ def test_verify_steps_refuses_a_chain_without_a_first_root_or_with_two_length_ar
     assert e.value.code == -1
     torch.cuda.synchronize()
     assert binding.mtv_device_error(tree) == 0
+
+
+def test_verify_steps_chain_replayed_from_a_cuda_graph():
+    """The chain of steps is one static sequence of launches: captured once into a CUDA graph and replayed, it gives
+    the results of the plain call (compared here) — no launch depends on anything the host would have to look at."""
+    B, H, V, Hq, Hkv, D, K, n_layers, n_steps = 2, 256, 2000, 8, 2, 128, 4, 2, 2
+    tb, tree = make_tree("rank_prior", K, (), 64)
+    T = tree.T
+    lens0 = torch.tensor([90, 33], dtype=torch.int32)
+    Lcap = int(lens0.max()) + n_steps * (K + 1) + T
+    seed = 211
+    hidden, W1, b1, W2, root = [t.to(DEV) for t in synth.head_inputs(B, H, V, K, seed)]
+    kc0 = [synth.normal_bf16(seed, 500 + l, (B, Hkv, Lcap, D)).to(DEV) for l in range(n_layers)]
+    vc0 = [synth.normal_bf16(seed, 600 + l, (B, Hkv, Lcap, D)).to(DEV) for l in range(n_layers)]
+    kd, vd = [t.clone() for t in kc0], [t.clone() for t in vc0]
+    q0 = torch.stack([synth.normal_bf16(seed, 700 + l, (B, T, Hq, D)) for l in range(n_layers)]).to(DEV)
+    kn = torch.stack([synth.normal_bf16(seed, 800 + l, (B, T, Hkv, D)) for l in range(n_layers)]).to(DEV)
+    vn = torch.stack([synth.normal_bf16(seed, 900 + l, (B, T, Hkv, D)) for l in range(n_layers)]).to(DEV)
+    logits = synth.normal_bf16(seed, 950, (B, T, V)).to(DEV)
+    sl = lens0.to(DEV)
+    ws = workspace(tree, B, H, V, Hq, Hkv, D, Lcap)
+    kp, vp = binding.cache_pointer_array(kd, DEV), binding.cache_pointer_array(vd, DEV)
+    kph, vph = binding.cache_pointer_array(kd), binding.cache_pointer_array(vd)
+    steps, appends, bufs = [], [], []
+    for s in range(n_steps):
+        dev = dict(hidden=hidden, W1=W1, b1=b1, W2=W2, q_layers=q0.clone(), logits=logits, seq_lens=sl,
+                   cand=_i32(B, tree.C), tree_tok=_i32(B, T),
+                   out_layers=torch.zeros(n_layers, B, T, Hq, D, dtype=torch.bfloat16, device=DEV),
+                   accept_len=_i32(B), best_path=_i32(B), acc_nodes=_i32(B, K + 1), acc_tok=_i32(B, K + 1),
+                   next_root=_i32(B), status=_i32(B), k_caches=kp, v_caches=vp, k_caches_host=kph, v_caches_host=vph, ws=ws)
+        if s == 0:
+            dev["root_tok"] = root
+        a = binding.StepArgs()
+        a.B, a.H, a.V, a.Hq, a.Hkv, a.D, a.n_layers, a.Lcap = B, H, V, Hq, Hkv, D, n_layers, Lcap
+        a.stride_b, a.stride_h, a.stride_t, a.scale = Hkv * Lcap * D, Lcap * D, D, 0.0
+        for name, t in dev.items():
+            setattr(a, name, t.data_ptr())
+        a.ws_bytes = ws.numel()
+        ap = binding.AppendArgs()
+        ap.k_new_layers, ap.v_new_layers, ap.rope_theta = kn.data_ptr(), vn.data_ptr(), 0.0
+        steps.append(a), appends.append(ap), bufs.append(dev)
+
+    def reset():
+        sl.copy_(lens0)
+        for l in range(n_layers):
+            kd[l].copy_(kc0[l]), vd[l].copy_(vc0[l])
+        for dev in bufs:
+            dev["q_layers"].copy_(q0)            # the append rotates the queries in place
+    names = ("cand", "tree_tok", "out_layers", "accept_len", "best_path", "acc_nodes", "acc_tok", "next_root")
+    reset()
+    binding.mtv_verify_steps(tree, steps, appends)
+    torch.cuda.synchronize()
+    want = [{n: dev[n].clone() for n in names} for dev in bufs]
+    want_sl, want_k = sl.clone(), [t.clone() for t in kd]
+    assert int(want_sl.min()) > int(lens0.min()) and binding.mtv_device_error(tree) == 0
+    # the same chain, captured and replayed
+    reset()
+    for dev in bufs:
+        for n in names:
+            dev[n].zero_()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            binding.mtv_verify_steps(tree, steps, appends, stream=side)
+    torch.cuda.current_stream().wait_stream(side)
+    reset()                                      # (capture launches nothing, but keep the state explicit)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert binding.mtv_device_error(tree) == 0
+    for dev, w_ in zip(bufs, want):
+        for n in names:
+            assert torch.equal(dev[n], w_[n]), n    # the same kernels on the same inputs: bit-identical
+    assert torch.equal(sl, want_sl)
+    for l in range(n_layers):
+        assert torch.equal(kd[l], want_k[l])
