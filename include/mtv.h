@@ -379,6 +379,12 @@ int mtv_verify_step_host(const mtv_tree_t *tree, const mtv_step_args *dev, const
  * keys_merge_shards: key_shards [n_shards][n] from lm_head_argmax on each slab (n = B * T) -> keys [n] for
  *   tree_accept_keys, the slab offsets folded into the index half; ties across slabs go to the lowest global id.
  */
+/* Per-node argmax keys of stored logits [B][T][V] (16-byte aligned base, as for tree_accept), in the form
+ * tree_accept_keys and keys_merge_shards read: keys [B*T]; ws as for tree_accept.  tree_accept(logits) equals
+ * node_argmax_keys followed by tree_accept_keys; a rank that holds the vocabulary slab [B][T][v_local] of the logits
+ * runs it on its slab, and keys_merge_shards over the gathered keys gives the keys of the whole vocabulary. */
+int node_argmax_keys(const mtv_tree_t *tree, int B, int V, const mtv_bf16 *logits, unsigned long long *keys,
+                     void *ws, size_t ws_bytes, void *stream);
 int heads_merge_shards(const mtv_tree_t *tree, int B, int n_shards, int v_slab, const int32_t *cand_shards,
                        const float *logit_shards, const int32_t *root_tok, int32_t *cand, float *cand_logit,
                        int32_t *tree_tok, void *ws, size_t ws_bytes, void *stream);

@@ -32,7 +32,7 @@ EXPORTS = ["tree_build_static", "tree_gen_cartesian", "tree_gen_rank_prior", "tr
            "tree_accept_static_scratch", "tree_accept_static_scratch_capacity", "tree_kv_append_rope",
            "lm_head_argmax", "tree_accept_keys", "mtv_selftest_wait_timeout", "tree_kv_append_rope_layers",
            "mtv_verify_steps", "mtv_debug_bounds_enabled", "heads_merge_shards", "attn_interleave_shards",
-           "keys_merge_shards"]
+           "keys_merge_shards", "node_argmax_keys"]
 
 
 class MtvError(RuntimeError):
@@ -119,6 +119,7 @@ def lib():
         L.heads_merge_shards.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.attn_interleave_shards.argtypes = [i32, i32, i32, i32, vp, vp, vp]
         L.keys_merge_shards.argtypes = [i32, i32, i32, vp, vp, vp]
+        L.node_argmax_keys.argtypes = [vp, i32, i32, vp, vp, vp, sz, vp]
         L.mtv_verify_steps.argtypes = [vp, C.POINTER(StepArgs), C.POINTER(AppendArgs), i32, vp]
         _lib = L
     return _lib
@@ -334,6 +335,13 @@ def attn_interleave_shards(gathered, out, stream=None):
     n, B, T, Hl, D = gathered.shape
     _check(lib().attn_interleave_shards(B * T, n, Hl, D, _ptr(gathered), _ptr(out), _stream(stream)),
            "attn_interleave_shards")
+
+
+def node_argmax_keys(tree, logits, keys, ws, stream=None):
+    """logits [B][T][V] bf16 -> keys [B*T] (int64 storage of the uint64 keys)."""
+    B, T, V = logits.shape
+    p, n = _ws(ws)
+    _check(lib().node_argmax_keys(tree.handle, B, V, _ptr(logits), _ptr(keys), p, n, _stream(stream)), "node_argmax_keys")
 
 
 def keys_merge_shards(v_slab, key_shards, keys, stream=None):

@@ -171,6 +171,41 @@ extern "C" int tree_accept(const mtv_tree_t *tree, int B, int V, const mtv_bf16 
     return MTV_OK;
 }
 
+// Per-node argmax keys of stored logits, in the form tree_accept_keys reads: what tree_accept computes before its path
+// scan.  A rank that holds a vocabulary slab of the logits calls this on its slab; keys_merge_shards then folds the
+// slab offsets in and takes the maximum over the ranks.
+namespace mtv {
+__global__ void argmax_keys_reduce_kernel(int rows, int ns, const unsigned long long *__restrict__ part,
+                                          unsigned long long *__restrict__ keys) {
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= rows) return;
+    unsigned long long best = 0;
+    for (int s = 0; s < ns; ++s) best = umax64(best, part[(size_t)r * ns + s]);
+    keys[r] = best;
+}
+}  // namespace mtv
+
+extern "C" int node_argmax_keys(const mtv_tree_t *tree, int B, int V, const mtv_bf16 *logits, unsigned long long *keys,
+                                void *ws, size_t ws_bytes, void *stream) {
+    using namespace mtv;
+    MTV_RANGE("node_argmax_keys");
+    if (!tree || !tree->on_device || !logits || !keys || !ws || B < 1 || V < 1) return MTV_ERR_INVALID_ARG;
+    if ((uintptr_t)logits & 15) return MTV_ERR_INVALID_ARG;
+    const AcceptWs L = accept_ws_layout(tree, B, V);
+    if (ws_bytes < L.total) return MTV_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    auto *part = reinterpret_cast<unsigned long long *>((char *)ws + L.part_off);
+    const int rows = B * tree->T;
+    {
+        TapScope tap(MTV_KERNEL_ARGMAX_PARTIAL, st);
+        node_argmax_partial_kernel<<<dim3(L.nsplit, rows), ARGMAX_THREADS, 0, st>>>(
+            V, reinterpret_cast<const __nv_bfloat16 *>(logits), part);
+    }
+    argmax_keys_reduce_kernel<<<(rows + 127) / 128, 128, 0, st>>>(rows, L.nsplit, part, keys);
+    MTV_CUDA_CHECK(cudaGetLastError());
+    return MTV_OK;
+}
+
 // Acceptance from per-node argmax keys (what lm_head_argmax leaves): the finish kernel alone, with
 // one key per node.
 extern "C" int tree_accept_keys(const mtv_tree_t *tree, int B, const unsigned long long *keys, const int32_t *tree_tok,

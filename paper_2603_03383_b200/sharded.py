@@ -7,7 +7,7 @@ over the vocabulary: rank r projects onto the slab ``[r * v_slab, min(V, (r + 1)
 and attends with their ``Hq / n`` query heads.  After each of the two, one all-gather brings every rank's result
 into a LOCAL buffer and a small kernel of the library merges the pieces (``heads_merge_shards``: same candidate
 order as on one device, so identical ids; ``attn_interleave_shards``; ``keys_merge_shards`` for the fused LM
-head).  No kernel is ever handed another GPU's memory; the collective is the group's backend (NCCL on GPUs).
+head and for the acceptance over vocabulary slabs of stored logits).  No kernel is ever handed another GPU's memory; the collective is the group's backend (NCCL on GPUs).
 
 This module holds the partition arithmetic and the collectives only; every step of the path itself runs in the
 library's kernels through ``binding``.  Everything is enqueued on the current torch stream (the collectives of
@@ -106,3 +106,16 @@ def lm_head_argmax_sharded(tree, p: ShardPlan, x, W_slab, keys, group=None):
     keys_l = torch.empty_like(keys)
     binding.lm_head_argmax(tree, x, W_slab, keys_l)
     binding.keys_merge_shards(p.v_slab, gather(keys_l, p.world, group), keys)
+
+
+def tree_accept_sharded(tree, p: ShardPlan, logits_slab, tree_tok, accept_len, best_path, acc_nodes, acc_tok, next_root, ws,
+                        group=None):
+    """logits_slab [B][T][v_local]: this rank's vocabulary slab of the base-model logits (contiguous).  Per-node argmax
+    of the slab, one all-gather of the (maximum, id) keys, the maximum over the ranks with the slab offsets folded in
+    (ties to the lowest global id), then the ordinary path scan: identical outputs on every rank."""
+    B, T, _ = logits_slab.shape
+    keys_l = torch.empty(B * T, dtype=torch.int64, device=logits_slab.device)
+    binding.node_argmax_keys(tree, logits_slab, keys_l, ws)
+    keys = torch.empty_like(keys_l)
+    binding.keys_merge_shards(p.v_slab, gather(keys_l, p.world, group), keys)
+    binding.tree_accept_keys(tree, B, keys, tree_tok, accept_len, best_path, acc_nodes, acc_tok, next_root)

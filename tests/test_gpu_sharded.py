@@ -161,3 +161,37 @@ def test_sharded_calls_with_a_group_of_one():
     torch.cuda.synchronize()
     assert torch.equal(cand.cpu(), cand_ref) and torch.equal(tt.cpu(), tt_ref)
     assert_close(out, ref.tree_attention(q, k, v, sl, tb["mask"]))
+
+
+@pytest.mark.parametrize("world,V", [(2, 1024), (4, 3001), (3, 777)])
+def test_accept_by_vocabulary_slab(world, V):
+    """Stored logits split by vocabulary slab: per-slab argmax keys, merged, give the acceptance of the whole vocabulary
+    (planted walks, natural ties across slabs included: the rows outside the walk are rounded N(0,1) draws)."""
+    K = 4
+    tb, tree = make_tree("rank_prior", K, (), 64)
+    B, T = 3, tree.T
+    g = torch.Generator().manual_seed(world)
+    cand = torch.stack([torch.randperm(V, generator=g)[:tb["C"]] for _ in range(B)]).to(torch.int32)
+    tree_tok = cand[:, torch.tensor(tb["tree_indices"])].contiguous()
+    logits, planted = synth.planted_logits(B, T, V, K, tree_tok, tb["parent"], tb["rank"], seed=40 + world, p_accept=(0.9, 0.5, 0.7))
+    logits[0, 5, V - 1] = logits[0, 5].max()          # an exact tie between a low id and the last id of the last slab
+    want = ref.tree_accept(ref.node_argmax(logits), tree_tok, tb)
+    ws = workspace(tree, B, 8, V, 0, 0, 0, 0)
+    key_all = torch.zeros(world, B * T, dtype=torch.int64, device=DEV)
+    for r in range(world):
+        p = sharded.plan(r, world, V, 48, 48)
+        binding.node_argmax_keys(tree, logits[:, :, p.v_lo:p.v_hi].contiguous().to(DEV), key_all[r], ws)
+    keys = torch.zeros(B * T, dtype=torch.int64, device=DEV)
+    binding.keys_merge_shards(p.v_slab, key_all, keys)
+    outs = dict(accept_len=_i32(B), best_path=_i32(B), acc_nodes=_i32(B, K + 1), acc_tok=_i32(B, K + 1), next_root=_i32(B))
+    binding.tree_accept_keys(tree, B, keys, tree_tok.to(DEV), outs["accept_len"], outs["best_path"], outs["acc_nodes"],
+                             outs["acc_tok"], outs["next_root"])
+    torch.cuda.synchronize()
+    am = (0xffffffff - (keys.cpu() & 0xffffffff)).to(torch.int32).reshape(B, T)
+    assert torch.equal(am, ref.node_argmax(logits))
+    for name, t in outs.items():
+        assert torch.equal(t.cpu(), want[name]), name
+    # the whole vocabulary in one call gives the same keys' indices, and tree_accept the same outputs
+    keys1 = torch.zeros(B * T, dtype=torch.int64, device=DEV)
+    binding.node_argmax_keys(tree, logits.to(DEV), keys1, ws)
+    assert torch.equal(keys1 & 0xffffffff, keys & 0xffffffff)
