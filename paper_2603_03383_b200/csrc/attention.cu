@@ -45,7 +45,7 @@ AttnWs attn_ws_layout(const mtv_tree *t, int B, int Hq, int Hkv, int D, int Lcap
     int ns = (int)(sm_count() / ctas);
     const int tiles = (Lcap + BN - 1) / BN;
     if (ns > tiles) ns = tiles;
-    if (ns < 1) ns = 1;
+    if (ns < 1 || tiles <= 4) ns = 1;   // a few tiles: one CTA per block writes the output itself (one launch instead of two)
     w.nsplit = ns;
     size_t off = 0;
     w.o_off = off;  off = align_up(off + (size_t)B * Hkv * ns * w.m_rows * D * sizeof(float), 256);
@@ -115,7 +115,9 @@ tree_attn_partial_kernel(const AttnParams p) {
     const int g = blockIdx.y / mblocks, mb = blockIdx.y % mblocks;
     const int b = blockIdx.z;
     const int L = p.seq_lens[b];
-    if (L + p.T > p.Lcap) return;     // reported by the combine kernel
+    if (p.nsplit == 1 && p.status && blockIdx.y == 0 && threadIdx.x == 0)   // no combine kernel follows: report here
+        p.status[b] = L + p.T > p.Lcap ? MTV_ERR_CAPACITY : MTV_OK;
+    if (L + p.T > p.Lcap) return;     // (with splits: reported by the combine kernel)
     const int n_keys = L + p.T;
     int t_begin, t_end;
     split_range(n_keys, p.nsplit, split, t_begin, t_end);
@@ -264,6 +266,18 @@ tree_attn_partial_kernel(const AttnParams p) {
     l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
 
+    if (p.nsplit == 1) {
+        // the only split of its block: normalise and write the output rows (row r = node * G + head-in-group)
+        const float inv0 = l0 > 0.f ? 1.f / l0 : 0.f, inv1 = l1 > 0.f ? 1.f / l1 : 0.f;
+        __nv_bfloat16 *o0 = p.out + (((size_t)b * p.T + r0 / p.G) * p.Hq + g * p.G + r0 % p.G) * D;
+        __nv_bfloat16 *o1 = p.out + (((size_t)b * p.T + r1 / p.G) * p.Hq + g * p.G + r1 % p.G) * D;
+#pragma unroll
+        for (int j = 0; j < D / 8; ++j) {
+            if (r0 < M) *reinterpret_cast<uint32_t *>(o0 + j * 8 + tq * 2) = pack_bf16(o[j][0] * inv0, o[j][1] * inv0);
+            if (r1 < M) *reinterpret_cast<uint32_t *>(o1 + j * 8 + tq * 2) = pack_bf16(o[j][2] * inv1, o[j][3] * inv1);
+        }
+        return;
+    }
     const size_t slab = (((size_t)b * p.Hkv + g) * p.nsplit + split) * p.m_rows;
     float *wo0 = p.ws_o + (slab + r0) * D, *wo1 = p.ws_o + (slab + r1) * D;
 #pragma unroll
@@ -361,7 +375,7 @@ extern "C" int tree_verify_attention(const mtv_tree_t *tree, int B, int Hq, int 
         if (D == 64) tree_attn_partial_kernel<64><<<grid, ATT_THREADS, smem, st>>>(p);
         else tree_attn_partial_kernel<128><<<grid, ATT_THREADS, smem, st>>>(p);
     }
-    {
+    if (Lw.nsplit > 1) {
         TapScope tap(MTV_KERNEL_ATTN_COMBINE, st);
         if (D == 64) tree_attn_combine_kernel<64><<<B * tree->T * Hq, 64, 0, st>>>(p);
         else tree_attn_combine_kernel<128><<<B * tree->T * Hq, 128, 0, st>>>(p);
