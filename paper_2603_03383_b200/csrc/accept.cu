@@ -1,6 +1,7 @@
 // Acceptance and token retrieval (Section 3.2, "Zero-Copy Retrieval"): per-node argmax
 // of the base-model logits, greedy longest-prefix match over the static paths, and the
 // gather of the accepted tokens through retrieve_indices — all on the device.
+#include <atomic>
 #include <cstdio>
 
 #include <cuda_bf16.h>
@@ -237,17 +238,20 @@ static __device__ __align__(256) unsigned char g_accept_scratch[ACCEPT_STATIC_SC
 // only a handle for the runtime, not an address a kernel could use, so the address is asked for
 // once per device (with that device current) and remembered.
 static int accept_scratch_address(unsigned long long **out) {
-    // (two host threads that meet on first use of a device both look the address up and store the same value)
-    static unsigned long long *cached[MTV_MAX_DEVICES] = {nullptr};
+    // (two host threads that meet on first use of a device both look the address up and store the same value;
+    // the slots are atomics so that neither ever reads a half-written pointer)
+    static std::atomic<unsigned long long *> cached[MTV_MAX_DEVICES];
     int dev = 0;
     MTV_CUDA_CHECK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= MTV_MAX_DEVICES) return MTV_ERR_UNSUPPORTED_SHAPE;
-    if (!cached[dev]) {
+    unsigned long long *addr = cached[dev].load(std::memory_order_acquire);
+    if (!addr) {
         void *ptr = nullptr;
         MTV_CUDA_CHECK(cudaGetSymbolAddress(&ptr, g_accept_scratch));
-        cached[dev] = reinterpret_cast<unsigned long long *>(ptr);
+        addr = reinterpret_cast<unsigned long long *>(ptr);
+        cached[dev].store(addr, std::memory_order_release);
     }
-    *out = cached[dev];
+    *out = addr;
     return MTV_OK;
 }
 

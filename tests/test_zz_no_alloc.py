@@ -57,6 +57,34 @@ def test_matches_tree_accept_on_two_calls_in_a_row():
         assert int(want[0].max()) >= 1              # the planted walks were found, not an all-zero coincidence
 
 
+def test_replays_from_a_cuda_graph():
+    """The call only enqueues two kernels: captured into a CUDA graph and replayed (no allocation, no synchronisation
+    inside), it gives the outputs of the plain call."""
+    K = 4
+    tb, tree = make_tree("rank_prior", K, (), 64)
+    B, V = 3, 9000
+    logits, tree_tok = _inputs(tb, B, tree.T, V, K, 21, (0.8, 0.4, 0.6))
+    want = _outputs(B, K)
+    binding.tree_accept_static_scratch(tree, logits, tree_tok, *want)     # also the first use on this device: outside capture
+    torch.cuda.synchronize()
+    got = _outputs(B, K)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            binding.tree_accept_static_scratch(tree, logits, tree_tok, *got, stream=side)
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(2):
+        for t in got:
+            t.fill_(-7)
+        graph.replay()
+        torch.cuda.synchronize()
+        for name, a, b in zip(NAMES, got, want):
+            assert torch.equal(a, b), name
+    assert int(want[0].max()) >= 1
+
+
 def test_refuses_logits_that_are_not_16_byte_aligned():
     """The row scan reads 16-byte chunks; a view that starts at an odd element is turned away on the host (an error
     code, no launch) by both entry points."""
