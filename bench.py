@@ -499,7 +499,8 @@ def run_sharded(args):
     local = int(os.environ.get("LOCAL_RANK", 0))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
+    use_dist = world > 1 or "RANK" in os.environ      # under torchrun the collectives are NCCL's even with one rank
+    if use_dist:
         dist.init_process_group("nccl", device_id=dev)
     w = synth.WORKLOADS[args.workload]
     n_layers = args.layers
@@ -572,12 +573,12 @@ def run_sharded(args):
         print(json.dumps({"metric": METRIC, "value": None, "unit": UNIT,
                           "error": "split step: attention differs from the unsplit step by %.3e on rank %d" % (err, rank)}))
         sys.exit(1)
+    sampler = ClockSampler(local)     # nvidia-smi takes a while to start: it runs from here to the end of the timed steps
+    if rank == 0:
+        sampler.start()
     for _ in range(W_steps):
         step()
     barrier()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     runs_ms = []
     for _ in range(max(1, args.repeats)):
         barrier()
@@ -643,7 +644,7 @@ def run_sharded(args):
                               "frac_of_measured": alg["step"] / ms_step / 1e6 / (pk["hbm_gbs"] * world)},
         }
         print(json.dumps(out))
-    if world > 1:
+    if use_dist:
         dist.destroy_process_group()
 
 
