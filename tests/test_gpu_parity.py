@@ -786,3 +786,48 @@ def test_verify_steps_chain_replayed_from_a_cuda_graph():
     assert torch.equal(sl, want_sl)
     for l in range(n_layers):
         assert torch.equal(kd[l], want_k[l])
+
+
+def _random_tree(g, K, T_target):
+    """A random ancestor-closed tree with up to T_target nodes (root included): nodes are added one at a time as the next
+    unused rank under a random existing node of depth < K."""
+    nodes, children = [()], {(): 0}
+    while len(nodes) < T_target:
+        cand = [n for n in nodes if len(n) < K and children[n] < 10]
+        if not cand:
+            break
+        parent = cand[int(torch.randint(0, len(cand), (1,), generator=g))]
+        child = parent + (children[parent],)
+        children[parent] += 1
+        children[child] = 0
+        nodes.append(child)
+    return [list(n) for n in nodes[1:]]
+
+
+@pytest.mark.parametrize("case", range(16))
+def test_attention_random_shapes(case):
+    """Seeded random problems: tree shape and size, head counts and head size, batch, prefix lengths (empty ones
+    included), cache capacity and a padded (strided) cache — the shapes no hand-picked case covers."""
+    from oracle import tree as otree
+    g = torch.Generator().manual_seed(1000 + case)
+    pick = lambda xs: xs[int(torch.randint(0, len(xs), (1,), generator=g))]
+    D = pick([64, 128, 128])
+    Hkv = pick([1, 2, 4, 8])
+    G = pick([1, 2, 4, 8])
+    Hq = Hkv * G
+    K = pick([1, 2, 3, 4, 5])
+    T_target = pick([2, 5, 17, 33, 64, 65, 97, 128])
+    nodes = _random_tree(g, K, T_target)
+    tb = otree.tables([tuple(n) for n in nodes], K)
+    tree = binding.tree_build_static(K, nodes, upload=True)
+    T = tree.T
+    assert T == tb["T"]
+    B = pick([1, 1, 2, 3, 5])
+    hi = pick([40, 300, 1300])
+    lens = [int(torch.randint(0, hi + 1, (1,), generator=g)) for _ in range(B)]
+    if case % 4 == 0:
+        lens[0] = 0
+    pad = pick([0, 0, 8, 40])
+    Lcap = max(lens) + T + pick([0, 1, 77])
+    _attention_case(tb, tree, B, Hq, Hkv, D, lens, seed=2000 + case, Lcap=Lcap, pad=pad)
+    assert binding.mtv_device_error(tree) == 0
