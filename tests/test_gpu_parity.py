@@ -831,3 +831,53 @@ def test_attention_random_shapes(case):
     Lcap = max(lens) + T + pick([0, 1, 77])
     _attention_case(tb, tree, B, Hq, Hkv, D, lens, seed=2000 + case, Lcap=Lcap, pad=pad)
     assert binding.mtv_device_error(tree) == 0
+
+
+@pytest.mark.parametrize("case", range(8))
+def test_heads_accept_compaction_random_trees(case):
+    """The integer part of a step on random trees (shapes the two generators never produce: uneven fan-out, leaves at
+    every depth): candidates and tree tokens from the heads, acceptance of planted walks, compaction of the accepted rows;
+    all bit-exact against the checker."""
+    from oracle import tree as otree
+    g = torch.Generator().manual_seed(3000 + case)
+    pick = lambda xs: xs[int(torch.randint(0, len(xs), (1,), generator=g))]
+    K = pick([2, 3, 4, 5])
+    nodes = _random_tree(g, K, pick([7, 20, 64, 100, 128]))
+    tb = otree.tables([tuple(n) for n in nodes], K)
+    tree = binding.tree_build_static(K, nodes, upload=True)
+    T, B = tree.T, pick([1, 2, 4, 7])
+    H, V = pick([64, 192, 520]), pick([300, 1001, 4096])
+    # ---- heads
+    seed, inp, _, cand_ref, cl_ref, tt_ref = oracle_heads_with_margin(B, H, V, K, tb, 3100 + case)
+    hidden, W1, b1, W2, root = [t.to(DEV) for t in inp]
+    ws = workspace(tree, B, H, V, 8, 2, 64, 64 + T)
+    cand, tt = _i32(B, tree.C), _i32(B, T)
+    binding.medusa_heads_topk(tree, hidden, W1, b1, W2, root, cand, None, tt, ws)
+    assert torch.equal(cand.cpu(), cand_ref) and torch.equal(tt.cpu(), tt_ref), seed
+    # ---- acceptance of planted walks
+    logits, planted = synth.planted_logits(B, T, V, K, tt_ref, tb["parent"], tb["rank"], seed, p_accept=(0.85, 0.5))
+    want = ref.tree_accept(ref.node_argmax(logits), tt_ref, tb)
+    assert torch.equal(want["accept_len"], planted)
+    outs = dict(accept_len=_i32(B), best_path=_i32(B), acc_nodes=_i32(B, K + 1), acc_tok=_i32(B, K + 1), next_root=_i32(B))
+    binding.tree_accept(tree, logits.to(DEV), tt, outs["accept_len"], outs["best_path"], outs["acc_nodes"], outs["acc_tok"],
+                        outs["next_root"], ws)
+    for name, t in outs.items():
+        assert torch.equal(t.cpu(), want[name]), name
+    # ---- compaction of those rows, two layers
+    Hkv, D = 2, 64
+    lens = [int(torch.randint(0, 60, (1,), generator=g)) for _ in range(B)]
+    Lcap = 64 + T
+    caches = [synth.normal_bf16(seed, 40 + l, (B, Hkv, Lcap, D)) for l in range(4)]
+    dev_c = [c.to(DEV) for c in caches]
+    kp, vp = binding.cache_pointer_array(dev_c[:2], DEV), binding.cache_pointer_array(dev_c[2:], DEV)
+    sl = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    status = _i32(B)
+    binding.kv_compact_accepted(tree, kp, vp, 2, B, Hkv, D, (Hkv * Lcap * D, Lcap * D, D), Lcap, sl, outs["accept_len"],
+                                outs["acc_nodes"], status=status)
+    torch.cuda.synchronize()
+    assert status.tolist() == [0] * B and binding.mtv_device_error(tree) == 0
+    for c, dc in zip(caches, dev_c):
+        want_c, new_len = ref.kv_compact(c, lens, want["accept_len"], want["acc_nodes"])
+        for b in range(B):
+            assert torch.equal(dc[b, :, :new_len[b]].cpu(), want_c[b, :, :new_len[b]])
+    assert torch.equal(sl.cpu(), torch.tensor(lens, dtype=torch.int32) + want["accept_len"] + 1)
