@@ -579,13 +579,30 @@ def run_sharded(args):
     for _ in range(W_steps):
         step()
     barrier()
+    run_step, launch = step, "stream launches"
+    if args.launch == "graph":
+        # the whole split step, collectives included, as one CUDA graph (every rank captures the same sequence)
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(graph, stream=side):
+                    step()
+            torch.cuda.current_stream().wait_stream(side)
+            for _ in range(2):
+                graph.replay()
+            run_step, launch = graph.replay, "one CUDA graph per step, replayed"
+        except Exception as e:      # a collective that cannot be captured: plain launches
+            launch = "stream launches (graph capture failed: %s)" % type(e).__name__
+        barrier()
     runs_ms = []
     for _ in range(max(1, args.repeats)):
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(K_steps):
-            step()
+            run_step()
         e1.record()
         barrier()
         runs_ms.append(max_over_ranks(e0.elapsed_time(e1), world, dev))
@@ -629,8 +646,8 @@ def run_sharded(args):
                        "parallelism": "one sequence set on %d GPU(s): heads by vocabulary slab (%d rows each), attention "
                                       "by KV head (%d of %d each), all-gather + merge kernel after each" % (
                                           world, pl.v_slab, pl.hkv_local, w.Hkv),
-                       "timing": "median of %d runs of %d steps (%s ms each), stream launches" % (
-                           len(runs_ms), K_steps, ", ".join("%.1f" % r for r in runs_ms)),
+                       "timing": "median of %d runs of %d steps (%s ms each), %s" % (
+                           len(runs_ms), K_steps, ", ".join("%.1f" % r for r in runs_ms), launch),
                        "l2": "inputs larger than L2: %.2f GB streamed per step over all ranks" % (alg["step"] / 1e9),
                        "collective_bytes_per_step_per_rank": gathered, "seed": w.seed, "context": PAPER_CONTEXT},
             "clocks": clocks,

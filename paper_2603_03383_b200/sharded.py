@@ -64,6 +64,23 @@ def plan(rank: int, world: int, V: int, Hq: int, Hkv: int, max_kd: int = 1, slab
                      rank * hkv_local)
 
 
+class Scratch:
+    """Buffers of the calls below, allocated on first use and reused (a hot loop then allocates nothing)."""
+
+    def __init__(self):
+        self._bufs = {}
+
+    def get(self, name, shape, dtype, device):
+        key = (name, tuple(shape), dtype, str(device))
+        buf = self._bufs.get(key)
+        if buf is None:
+            buf = self._bufs[key] = torch.empty(tuple(shape), dtype=dtype, device=device)
+        return buf
+
+
+_default_scratch = Scratch()
+
+
 def gather(t: torch.Tensor, world: int, group=None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
     """All ranks' `t` (same shape everywhere) as one local tensor ``[world, *t.shape]``."""
     t = t.contiguous()
@@ -77,45 +94,52 @@ def gather(t: torch.Tensor, world: int, group=None, out: Optional[torch.Tensor] 
 
 
 def medusa_heads_topk_sharded(tree, p: ShardPlan, hidden, W1, b1, W2_slab, root_tok, cand, cand_logit, tree_tok, ws,
-                              group=None):
+                              group=None, scratch: Optional[Scratch] = None):
     """W2_slab [K][v_local][H]: this rank's rows of every head.  cand, cand_logit, tree_tok as medusa_heads_topk
     on the whole vocabulary writes them (identical on every rank)."""
-    B = hidden.shape[0]
+    B, dev = hidden.shape[0], hidden.device
+    sc = scratch or _default_scratch
     assert W2_slab.shape[1] == p.v_local
-    cand_l = torch.empty(B, tree.C, dtype=torch.int32, device=hidden.device)
-    logit_l = torch.empty(B, tree.C - 1, dtype=torch.float32, device=hidden.device)
-    tt_l = torch.empty(B, tree.T, dtype=torch.int32, device=hidden.device)
+    cand_l = sc.get("cand_l", (B, tree.C), torch.int32, dev)
+    logit_l = sc.get("logit_l", (B, tree.C - 1), torch.float32, dev)
+    tt_l = sc.get("tt_l", (B, tree.T), torch.int32, dev)
     binding.medusa_heads_topk(tree, hidden, W1, b1, W2_slab, root_tok, cand_l, logit_l, tt_l, ws)
-    cand_all = gather(cand_l, p.world, group)
-    logit_all = gather(logit_l, p.world, group)
+    cand_all = gather(cand_l, p.world, group, sc.get("cand_all", (p.world, B, tree.C), torch.int32, dev))
+    logit_all = gather(logit_l, p.world, group, sc.get("logit_all", (p.world, B, tree.C - 1), torch.float32, dev))
     binding.heads_merge_shards(tree, p.v_slab, cand_all, logit_all, root_tok, cand, cand_logit, tree_tok, ws)
 
 
 def tree_verify_attention_sharded(tree, p: ShardPlan, q_local, k_local, v_local, seq_lens, out, ws, scale=0.0,
-                                  status=None, group=None, Lcap=None):
+                                  status=None, group=None, Lcap=None, scratch: Optional[Scratch] = None):
     """q_local [B][T][hq_local][D], k_local / v_local [B][hkv_local][Lcap][D]: this rank's heads.  out
     [B][T][Hq][D]: all heads, identical on every rank."""
-    out_l = torch.empty_like(q_local)
+    sc = scratch or _default_scratch
+    out_l = sc.get("out_l", q_local.shape, q_local.dtype, q_local.device)
     binding.tree_verify_attention(tree, q_local, k_local, v_local, seq_lens, out_l, ws, scale=scale, status=status,
                                   Lcap=Lcap)
-    binding.attn_interleave_shards(gather(out_l, p.world, group), out)
+    gathered = sc.get("out_all", (p.world,) + tuple(q_local.shape), q_local.dtype, q_local.device)
+    binding.attn_interleave_shards(gather(out_l, p.world, group, gathered), out)
 
 
-def lm_head_argmax_sharded(tree, p: ShardPlan, x, W_slab, keys, group=None):
+def lm_head_argmax_sharded(tree, p: ShardPlan, x, W_slab, keys, group=None, scratch: Optional[Scratch] = None):
     """W_slab [v_local][H]: this rank's rows of the LM head.  keys [B*T]: the input of tree_accept_keys."""
-    keys_l = torch.empty_like(keys)
+    sc = scratch or _default_scratch
+    keys_l = sc.get("keys_l", keys.shape, keys.dtype, keys.device)
     binding.lm_head_argmax(tree, x, W_slab, keys_l)
-    binding.keys_merge_shards(p.v_slab, gather(keys_l, p.world, group), keys)
+    keys_all = sc.get("keys_all", (p.world,) + tuple(keys.shape), keys.dtype, keys.device)
+    binding.keys_merge_shards(p.v_slab, gather(keys_l, p.world, group, keys_all), keys)
 
 
 def tree_accept_sharded(tree, p: ShardPlan, logits_slab, tree_tok, accept_len, best_path, acc_nodes, acc_tok, next_root, ws,
-                        group=None):
+                        group=None, scratch: Optional[Scratch] = None):
     """logits_slab [B][T][v_local]: this rank's vocabulary slab of the base-model logits (contiguous).  Per-node argmax
     of the slab, one all-gather of the (maximum, id) keys, the maximum over the ranks with the slab offsets folded in
     (ties to the lowest global id), then the ordinary path scan: identical outputs on every rank."""
     B, T, _ = logits_slab.shape
-    keys_l = torch.empty(B * T, dtype=torch.int64, device=logits_slab.device)
+    sc, dev = scratch or _default_scratch, logits_slab.device
+    keys_l = sc.get("akeys_l", (B * T,), torch.int64, dev)
     binding.node_argmax_keys(tree, logits_slab, keys_l, ws)
-    keys = torch.empty_like(keys_l)
-    binding.keys_merge_shards(p.v_slab, gather(keys_l, p.world, group), keys)
+    keys = sc.get("akeys", (B * T,), torch.int64, dev)
+    keys_all = sc.get("akeys_all", (p.world, B * T), torch.int64, dev)
+    binding.keys_merge_shards(p.v_slab, gather(keys_l, p.world, group, keys_all), keys)
     binding.tree_accept_keys(tree, B, keys, tree_tok, accept_len, best_path, acc_nodes, acc_tok, next_root)
