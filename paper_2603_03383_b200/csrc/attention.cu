@@ -352,7 +352,7 @@ extern "C" int tree_verify_attention(const mtv_tree_t *tree, int B, int Hq, int 
     p.nsplit = Lw.nsplit; p.m_rows = Lw.m_rows;
     cudaStream_t st = (cudaStream_t)stream;
     if (Lw.use_tc && scale >= 0.f) {
-        // tcgen05 path: head_dim 128, query groups of 1/2/4/8 heads; one launch
+        // tcgen05 path: head_dim 128, query groups of up to 8 heads; one launch
         TapScope tap(MTV_KERNEL_ATTN_PARTIAL, st);
         const int rc = launch_tree_attn_tc(tree, B, Hq, Hkv, p.q, p.k, p.v, stride_b, stride_h, stride_t, Lcap, seq_lens,
                                            p.scale_log2, p.out, status, p.ws_o, p.ws_ml,

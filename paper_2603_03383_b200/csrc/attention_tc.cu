@@ -1,7 +1,8 @@
 // Tree attention on the 5th-generation tensor cores (Section 3.2 / Fig. 2(b)), head_dim 128.
 //
 // A pair of CTAs (a cluster of two) owns up to 256 query rows — the (node, head-in-group) rows that
-// share one KV head — and every nsplit-th 128-key group of the sequence.  The two CTAs form one
+// share one KV head: 128 / G whole tree nodes per CTA for a group of G <= 8 query heads (when G does not
+// divide 128 the last rows of a CTA's tile stay unused) — and every nsplit-th 128-key group of the sequence.  The two CTAs form one
 // tcgen05 CTA pair: each keeps 128 of the query rows, its own S / P / O in tensor memory and its own
 // softmax warps, and each loads HALF of every K and V group from global memory (K: 64 of the 128 keys;
 // V: 64 of the 128 columns), so a K/V byte crosses from L2 to the SMs once per 256 query rows.  The
@@ -113,7 +114,8 @@ struct TcParams {
     const int32_t *order;  // [B] sequences by descending length, or null: grid index z -> sequence
     int32_t *dev_error;
     float scale_log2;
-    int T, G, Hq, Hkv, Lcap, nsplit, n_blk, M_rows;
+    int T, G, Hq, Hkv, Lcap, nsplit, n_blk;
+    int npc, R;   // tree nodes per CTA (128 / G) and the query rows they fill (npc * G <= 128: the other rows of the tile idle)
 };
 
 // 128-byte-swizzled shared-memory operand descriptor.
@@ -252,7 +254,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     int b = p.order ? p.order[blockIdx.z] : blockIdx.z;
     if (!MTV_INDEX_OK(b, gridDim.z, p.dev_error)) b = blockIdx.z;   // (both CTAs of a pair read the same entry)
     const int L = p.seq_lens[b];
-    const int rows0 = blk * 256 + (int)rank * 128;   // first row of this CTA inside the (sequence, KV head) block
+    // This CTA's query rows: row = (node - node0) * G + head-in-group for its npc nodes; with a group size that does not
+    // divide 128 the last 128 - R rows of the tile belong to nobody (zeroed, computed, never written out).
+    const int node0 = (blk * 2 + (int)rank) * p.npc;
+    auto valid_row = [&](int lrow) { return lrow < p.R && node0 + lrow / p.G < p.T; };
     auto tile_of = [&](int j) { return split + j * p.nsplit; };
     auto issue_k = [&](int j) {
         const int s = j % TC_STAGES;
@@ -272,9 +277,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
         // are split, split + nsplit, ...; past the end of the cache a copy delivers zeros), so they are requested while
         // the length is still on its way; they only touch this CTA's own shared memory and barriers.
         issue_k(0);
-        ptx::mbar_arrive_expect_tx(bar(BAR_QFULL), TC_Q_BYTES);
+        ptx::mbar_arrive_expect_tx(bar(BAR_QFULL), (uint32_t)p.R * 256u);
         for (int half = 0; half < 2; ++half)
-            ptx::tma_load_4d(q_smem + half * TC_Q_HALF, &q_map, bar(BAR_QFULL), half * 64, g * p.G, rows0 / p.G, b);
+            ptx::tma_load_4d(q_smem + half * TC_Q_HALF, &q_map, bar(BAR_QFULL), half * 64, g * p.G, node0, b);
         issue_k(1);
         issue_v(0);
         issue_v(1);
@@ -286,7 +291,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     const int tiles = (n_keys + TC_BN - 1) / TC_BN;
     // key tiles split, split + nsplit, ... : the splits of a query block read neighbouring tiles at the same time
     const int cnt = over || split >= tiles ? 0 : (tiles - split + p.nsplit - 1) / p.nsplit;
-    const bool have_rows = rows0 < p.M_rows;
+    const bool have_rows = node0 < p.T;
     if (warp != TC_TMA_WARP) ptx::cluster_wait();   // the producer first requests this CTA's own tiles
 
     // A wait that ran out: flag both CTAs of the pair and raise the sticky error.
@@ -350,7 +355,19 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
             if (j == 0) {
                 ok = ptx::mbar_wait(bar(BAR_QFULL), 0);
                 if (!ok) break;
-                if (lane == 0) ptx::mbar_arrive_remote(lead(BAR_QREADY));
+                if (p.R < 128) {
+                    // the tile's unused rows hold whatever shared memory held: clear them (a row stays in its own 128
+                    // bytes of each half under the swizzle), so that the scores of those rows are plain zeros
+                    for (int e = p.R * 8 + lane; e < 128 * 8; e += 32) {
+                        reinterpret_cast<uint4 *>(gbase)[e] = make_uint4(0u, 0u, 0u, 0u);
+                        reinterpret_cast<uint4 *>(gbase + TC_Q_HALF)[e] = make_uint4(0u, 0u, 0u, 0u);
+                    }
+                    ptx::fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive_remote_release(lead(BAR_QREADY));
+                } else if (lane == 0) {
+                    ptx::mbar_arrive_remote(lead(BAR_QREADY));
+                }
             }
             ok = ptx::mbar_wait(bar(BAR_VFULL + s), par);
             if (!ok) break;
@@ -447,9 +464,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
         // Thread (row, st) owns query row `row` in stream st: keys [64 st, 64 st + 64) of every group.
         const int qd = warp & 3, st = warp >> 2;
         const int row = qd * 32 + lane;
-        const int r = rows0 + row;
         uint64_t alo = 0, ahi = 0;
-        if (r < p.M_rows) { alo = p.anc[(r / p.G) * 2]; ahi = p.anc[(r / p.G) * 2 + 1]; }
+        if (valid_row(row)) { alo = p.anc[(node0 + row / p.G) * 2]; ahi = p.anc[(node0 + row / p.G) * 2 + 1]; }
         const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
         const uint32_t t_s = tmem + lane_base + TM_S + st * 64;   // + 128 for the odd groups; P goes over its first 32 columns
         const uint32_t t_o = tmem + lane_base + TM_O + st * 128;
@@ -611,8 +627,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
                 }
             }
         }
-        auto out_ptr = [&](int rr) {   // the 128 output values of query-block row rr
-            const int node = rr / p.G, hq = g * p.G + rr % p.G;
+        auto out_ptr = [&](int lrow) {   // the 128 output values of this CTA's row lrow
+            const int node = node0 + lrow / p.G, hq = g * p.G + lrow % p.G;
             return p.out + (((size_t)b * p.T + node) * p.Hq + hq) * 128;
         };
         const int grp = blockIdx.z * gridDim.y + blockIdx.y;
@@ -638,7 +654,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
 #pragma unroll
                 for (int it = 0; it < 8; ++it) {
                     const int srow = qd * 32 + st * 16 + it * 2 + hs;
-                    if (rows0 + srow < p.M_rows) *reinterpret_cast<uint4 *>(out_ptr(rows0 + srow) + ch * 8) = v[it];
+                    if (valid_row(srow)) *reinterpret_cast<uint4 *>(out_ptr(srow) + ch * 8) = v[it];
                 }
             } else {
                 uint4 *dst = reinterpret_cast<uint4 *>(p.ws_o + ((slab0 + split) * 256 + slab_row0 + qd * 32 + st * 16 + hs) * 128 + ch * 8);
@@ -675,8 +691,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
             for (int rl0 = warp * 2; rl0 < n_my; rl0 += 2 * TC_SOFTMAX_WARPS) {   // warp-uniform trip count: shuffles inside
                 const bool mine = rl0 + hs < n_my;
                 const int rl = mine ? rl0 + hs : rl0;            // the odd half warp may have no row: it repeats its neighbour's loads
-                const int srow = slab_row0 + row_begin + rl;     // row inside a slab
-                const int rr = blk * 256 + srow;                 // row inside the (sequence, KV head) block
+                const int lrow = row_begin + rl;                 // row of this CTA
+                const int srow = slab_row0 + lrow;               // row inside a slab
                 const __nv_bfloat16 *src = p.ws_o + (slab0 * 256 + srow) * 128 + ch * 8;
                 float acc[8];
 #pragma unroll
@@ -719,8 +735,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
                 }
                 if (warp == 0) TRACE(43);   // rows of all splits arrived and combined
                 const float inv = wsum > 0.f ? 1.f / wsum : 0.f;
-                if (mine && rr < p.M_rows)
-                    *reinterpret_cast<uint4 *>(out_ptr(rr) + ch * 8) =
+                if (mine && valid_row(lrow))
+                    *reinterpret_cast<uint4 *>(out_ptr(lrow) + ch * 8) =
                         make_uint4(pack2_bf16(acc[0] * inv, acc[1] * inv), pack2_bf16(acc[2] * inv, acc[3] * inv),
                                    pack2_bf16(acc[4] * inv, acc[5] * inv), pack2_bf16(acc[6] * inv, acc[7] * inv));
             }
@@ -827,7 +843,7 @@ __global__ void attn_order_kernel(const int32_t *seq_lens, int B, int32_t *order
 }
 constexpr int TC_ORDER_MAX_B = 2048;
 
-bool attn_tc_eligible(int D, int G) { return D == 128 && (G == 1 || G == 2 || G == 4 || G == 8); }
+bool attn_tc_eligible(int D, int G) { return D == 128 && G >= 1 && G <= 8; }
 
 static int tc_prepare() {
     static PerDeviceOnce once;
@@ -843,7 +859,8 @@ static int tc_prepare() {
 // per SM), at most one per key tile, at most TC_MAX_SPLITS.  More than one split needs two merge counters
 // per query block.
 int attn_tc_plan(int T, int G, int B, int Hkv, int Lcap, int *n_blk_out) {
-    const int n_blk = (T * G + 255) / 256;
+    const int npc = 128 / G;                      // tree nodes per CTA; a pair takes 2 npc
+    const int n_blk = (T + 2 * npc - 1) / (2 * npc);
     const long base = (long)B * Hkv * n_blk;
     const int tiles = (Lcap + TC_BN - 1) / TC_BN;
     long ns = (sm_count() / 2) / base;
@@ -880,7 +897,8 @@ int launch_tree_attn_tc(const mtv_tree *tree, int B, int Hq, int Hkv, const __nv
     p.scale_log2 = scale_log2;
     p.T = T; p.G = G; p.Hq = Hq; p.Hkv = Hkv; p.Lcap = Lcap;
     p.nsplit = attn_tc_plan(T, G, B, Hkv, Lcap, &p.n_blk);
-    p.M_rows = T * G;
+    p.npc = 128 / G;
+    p.R = p.npc * G;
     p.order = nullptr;
     if (p.nsplit == 1 && B > 1 && B <= TC_ORDER_MAX_B && (long)B * Hkv * p.n_blk > sm_count() / 2 && ws_order) {
         attn_order_kernel<<<(B + 255) / 256, 256, 0, stream>>>(seq_lens, B, ws_order);

@@ -104,6 +104,11 @@ def test_attention_prefix_lengths_tiny_tree(L):
     ("cartesian", 1, (1,), 0, 4, 4, 64, [50]),                     # T = 2, no grouping
     ("cartesian", 1, (), 0, 2, 1, 128, [40, 3]),                   # root-only tree
     ("cartesian", 3, (4, 2, 2), 0, 8, 2, 64, [128]),               # the tiny configuration
+    ("rank_prior", 4, (), 64, 28, 4, 128, [3000]),                 # groups of 7 heads (18 nodes per CTA, 126 of 128 rows), key splits
+    ("rank_prior", 5, (), 128, 21, 3, 128, [200, 0, 77]),          # groups of 7, four row blocks, ragged batch
+    ("rank_prior", 4, (), 65, 12, 4, 128, [517, 64]),              # groups of 3
+    ("rank_prior", 4, (), 64, 10, 2, 128, [1100]),                 # groups of 5 (25 nodes per CTA, 125 rows)
+    ("cartesian", 2, (3, 2), 0, 12, 2, 128, [90, 300, 5]),         # groups of 6, a ten-node tree
 ])
 def test_attention_shapes(kind, K, topk, T, Hq, Hkv, D, lens):
     tb, tree = make_tree(kind, K, topk, T)
@@ -804,7 +809,7 @@ def _random_tree(g, K, T_target):
     return [list(n) for n in nodes[1:]]
 
 
-@pytest.mark.parametrize("case", range(16))
+@pytest.mark.parametrize("case", range(20))
 def test_attention_random_shapes(case):
     """Seeded random problems: tree shape and size, head counts and head size, batch, prefix lengths (empty ones
     included), cache capacity and a padded (strided) cache — the shapes no hand-picked case covers."""
@@ -814,6 +819,9 @@ def test_attention_random_shapes(case):
     D = pick([64, 128, 128])
     Hkv = pick([1, 2, 4, 8])
     G = pick([1, 2, 4, 8])
+    if case >= 16:
+        G = [3, 5, 6, 7][case - 16]              # group sizes that do not divide the 128 rows of a tile
+        D, Hkv = 128, pick([1, 2, 4])
     Hq = Hkv * G
     K = pick([1, 2, 3, 4, 5])
     T_target = pick([2, 5, 17, 33, 64, 65, 97, 128])
