@@ -65,7 +65,7 @@ def peaks():
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
 # profiles/, keyed by tap name, with the hash of the kernel's source at capture time: a changed kernel reports null.
 NCU_TRAFFIC = {
-    "attn_partial": ("attention_tc.cu", "693ab104544828f5", 34.4128e6 + 0.0003e6),
+    "attn_partial": ("attention_tc.cu", "3b39f055e83c8c7d", 34.4122e6 + 0.0003e6),
     "heads_vocab_topk": ("heads.cu", "914e411d83fc386f", 4.2995e9),
     "lm_head_argmax": ("lm_head.cu", "8eac35b20edf1166", 1.0795e9),
 }
